@@ -1,0 +1,187 @@
+/*
+ * fastpool - C ABI of the multi-LoRA forward step over one unified LoRA/KV block pool (sm_100a).
+ *
+ * The paper (Section 4.3, "Unified Caching Pool for LoRAs and KVs") cuts HBM and main memory into
+ * blocks of one size, keeps LoRA adapters (partitioned block-wise along the rank dimension) and KV
+ * caches in the same blocks, addresses them through block tables, and swaps whole blocks between
+ * the two memories on a side stream.  This library is that pool plus the three computations that
+ * run over it: the segmented LoRA projection (Eq. 1, Eq. 2, Section 2.1), paged prefill/decode
+ * attention over [cached prefix || new tokens] (Section 2.1, Section 4.2), and the block swap
+ * (Section 4.3 "Asynchronous Swapping-in/out").
+ *
+ * Conventions
+ *  - Every function returns an int status: FL_OK or a negative FL_E* code.  Nothing throws or aborts.
+ *  - "device pointer" = memory of the pool's GPU, owned by the caller, at least 16-byte aligned;
+ *    "host pointer" = ordinary host memory.  The library never frees caller memory.
+ *  - bf16 values are passed as raw 16-bit patterns (fl_bf16).  Head dimension is 128.
+ *  - Kernel launches are asynchronous on the given stream; a status of FL_OK means "enqueued".
+ *    Kernels never trap: a block id or token position outside the pool makes the thread skip the
+ *    access and set a sticky flag that fl_pool_status reports.
+ *  - A pool belongs to one device; calls on one pool from several host threads must be serialised
+ *    by the caller.
+ */
+#ifndef FASTPOOL_H
+#define FASTPOOL_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct fl_pool fl_pool;
+typedef uint16_t fl_bf16;
+typedef struct CUstream_st* fl_stream;   /* a cudaStream_t; NULL = the default stream */
+typedef struct CUevent_st* fl_event;     /* a cudaEvent_t */
+
+enum {
+  FL_OK = 0,
+  FL_EINVAL = -1,   /* bad argument (null pointer, misaligned size, shape the kernels do not cover) */
+  FL_ENOMEM = -2,   /* not enough free blocks (the paper's "HBM is full"), or workspace too small */
+  FL_EBADID = -3,   /* block id out of range / not allocated / freed twice; unknown adapter id */
+  FL_EBUSY = -4,    /* reserved */
+  FL_ECUDA = -5,    /* a CUDA call failed; fl_last_cuda_error gives the cudaError_t */
+  FL_ETIMEOUT = -6  /* fl_swap_wait: the copies did not finish before the deadline */
+};
+
+#define FL_HEAD_DIM 128
+#define FL_MAX_MATS 8
+#define FL_MAX_RANK 64
+#define FL_MAX_LORA_ID (1 << 20)
+
+/* Shape of one LoRA-carrying projection: A is [d_in, rank], B is [rank, d_out]. */
+typedef struct { int32_t d_in, d_out; } fl_lora_shape;
+
+/* Sticky device-side flags and counters, see fl_pool_status. */
+typedef struct {
+  uint32_t device_flags;        /* bit 0: block id out of range seen by a kernel; bit 1: token position
+                                   beyond its block table; bit 2: adapter id not registered;
+                                   bit 3: a bounded wait inside a kernel gave up */
+  uint32_t blocks_used, blocks_free, host_blocks_used, host_blocks_free;
+  uint32_t lora_blocks;         /* device blocks referenced by registered adapters */
+  uint64_t bytes_swapped_in, bytes_swapped_out;
+} fl_status;
+
+/* ---------------------------------------------------------------- pool (Section 4.3)
+ * Allocates one device slab of n_blocks * block_bytes on `device` and one pinned host slab of
+ * n_host_blocks * block_bytes ("both HBM and main memory are partitioned into memory blocks of the
+ * same size").  block_bytes must be a multiple of 512.  The pool owns both slabs until
+ * fl_pool_destroy.  FL_ECUDA if an allocation fails. */
+int fl_pool_create(fl_pool** out, size_t block_bytes, uint32_t n_blocks, uint32_t n_host_blocks, int device);
+int fl_pool_destroy(fl_pool* pool);
+
+/* Block allocator.  The paper only says freed blocks are recycled for future allocations; the order
+ * used here: each memory has a LIFO stack, a fresh pool hands out 0, 1, 2, ..., fl_block_free pushes
+ * ids in list order.  Both calls are all-or-nothing: FL_ENOMEM (alloc) or FL_EBADID (free of an id
+ * that is out of range, not allocated, or listed twice) leave the pool unchanged.  ids: host pointer. */
+int fl_block_alloc(fl_pool* pool, uint32_t n, uint32_t* ids);
+int fl_block_free(fl_pool* pool, uint32_t n, const uint32_t* ids);
+int fl_host_block_alloc(fl_pool* pool, uint32_t n, uint32_t* ids);
+int fl_host_block_free(fl_pool* pool, uint32_t n, const uint32_t* ids);
+
+/* Base addresses of the two slabs (block i starts at base + i * block_bytes). */
+void* fl_pool_device_base(fl_pool* pool);
+void* fl_pool_host_base(fl_pool* pool);
+
+/* Synchronous copy of one DEVICE block to / from ordinary host memory (block_bytes bytes); for
+ * inspection and tests, not part of the hot path.  FL_EBADID if id >= n_blocks. */
+int fl_block_read(fl_pool* pool, uint32_t id, void* dst_host);
+int fl_block_write(fl_pool* pool, uint32_t id, const void* src_host);
+
+/* Copies the free stack (bottom first; the last entry is handed out next) into `free_ids` (host pointer,
+ * capacity `cap`) and writes its length to *n_free.  host != 0 selects the host memory's stack.
+ * Used to compare allocator state bit for bit. */
+int fl_pool_snapshot(fl_pool* pool, int host, uint32_t* free_ids, uint32_t cap, uint32_t* n_free);
+/* Reads the sticky device flags (synchronises the device) and the counters.  clear != 0 resets the flags. */
+int fl_pool_status(fl_pool* pool, fl_status* out, int clear);
+int fl_last_cuda_error(fl_pool* pool);
+
+/* ---------------------------------------------------------------- adapters (Section 4.3)
+ * "We perform block-wise partitioning of LoRAs along the rank dimension": an adapter is stored as
+ * rank-rows.  Row p of A_m is A_m[:, p] (d_in values), row p of B_m is B_m[p, :] (d_out values); rows
+ * are taken in the order A_0, B_0, A_1, B_1, ...; rows of equal width form one class (classes in order
+ * of first appearance); a class is a packed sequence of rows that never straddle a block, with
+ * rows_per_block = block_bytes / (2 * width); class c starts at the table entry after the blocks of
+ * the classes before it.  Row g of a class is in table[class_base + g / rows_per_block] at byte
+ * (g % rows_per_block) * 2 * width.  Every width must be a multiple of 8 and fit in one block.
+ *
+ * fl_lora_blocks: number of table entries (= blocks) such an adapter needs -> *n_table. */
+int fl_lora_blocks(size_t block_bytes, int32_t rank, const fl_lora_shape* mats, int n_mats, uint32_t* n_table);
+/* Writes the adapter into HOST pool blocks in that layout; weights reach HBM only through fl_swap_in
+ * (the paper loads adapters from main memory).  A[m]: host pointer, [d_in, rank] row-major;
+ * B[m]: host pointer, [rank, d_out] row-major; host_blocks: n_table allocated host block ids. */
+int fl_lora_pack_host(fl_pool* pool, int32_t rank, const fl_lora_shape* mats, int n_mats,
+                      const fl_bf16* const* A, const fl_bf16* const* B,
+                      const uint32_t* host_blocks, uint32_t n_table);
+/* Registers adapter `lora_id` (0 <= id < FL_MAX_LORA_ID, 1 <= rank <= FL_MAX_RANK, n_mats <= FL_MAX_MATS)
+ * whose rows live in the DEVICE blocks block_table[0..n_table) (host pointer; copied into the device-side
+ * adapter directory; the blocks stay allocated by the caller).  All adapters of a pool share the
+ * projection shapes `mats` (ranks may differ): the first registration fixes them, a later mismatch
+ * is FL_EINVAL.  Re-registering an id replaces it.  Synchronous with respect to the device. */
+int fl_lora_register(fl_pool* pool, int32_t lora_id, int32_t rank, const fl_lora_shape* mats, int n_mats,
+                     const uint32_t* block_table, uint32_t n_table);
+int fl_lora_unregister(fl_pool* pool, int32_t lora_id);
+
+/* ---------------------------------------------------------------- LoRA projection (Eq. 1, Eq. 2; Section 2.1 SGMV)
+ * For every segment s (tokens seg_indptr[s] .. seg_indptr[s+1]) with adapter i = lora_ids[s]:
+ *     y[t, :] += scale * (x[t, :] A_i) B_i        (A_i, B_i = projection `mat_index` of adapter i)
+ * y already holds the base projection x W; lora_ids[s] < 0 leaves the segment untouched.
+ * x: device [n_tokens, d_in] bf16 row-major; y: device [n_tokens, d_out] bf16 row-major, updated in place
+ * (fp32 accumulation, one bf16 rounding of the sum).  seg_indptr [n_seg+1], lora_ids [n_seg]: device int32.
+ * workspace: device scratch of at least fl_lora_sgmv_workspace(n_tokens, n_mats) bytes, contents
+ * irrelevant before and after; calls that share a workspace must be ordered on one stream.
+ * The _multi form applies n_mats projections that share x (q, k, v) in one pass: ys[j] and
+ * mat_indices[j] are HOST arrays of device pointers / indices. */
+size_t fl_lora_sgmv_workspace(int n_tokens, int n_mats);
+int fl_lora_sgmv(fl_pool* pool, fl_bf16* y, const fl_bf16* x, int mat_index,
+                 const int32_t* seg_indptr, const int32_t* lora_ids, int n_seg, int n_tokens,
+                 float scale, void* workspace, size_t workspace_bytes, fl_stream stream);
+int fl_lora_sgmv_multi(fl_pool* pool, fl_bf16* const* ys, const fl_bf16* x, const int* mat_indices, int n_mats,
+                       const int32_t* seg_indptr, const int32_t* lora_ids, int n_seg, int n_tokens,
+                       float scale, void* workspace, size_t workspace_bytes, fl_stream stream);
+
+/* ---------------------------------------------------------------- KV store (Section 4.3: new KV stays in HBM blocks)
+ * Writes the new tokens' K and V into the pool.  Request i owns tokens req_indptr[i] .. req_indptr[i+1]
+ * of k_new / v_new (device, [n_tokens, n_kv_heads, 128] bf16); its token j goes to logical position
+ * prefix_lens[i] + j, i.e. block kv_tbl[kv_tbl_indptr[i] + pos / bt], slot pos % bt, where
+ * bt = block_bytes / (2 * n_kv_heads * 128 * 2).  In-block layout: [K|V][kv_head][token][128] bf16.
+ * req_indptr, kv_tbl_indptr [n_req+1], prefix_lens [n_req]: device int32; kv_tbl: device uint32.
+ * The tables must already cover prefix_len + new tokens. */
+int fl_kv_append(fl_pool* pool, const fl_bf16* k_new, const fl_bf16* v_new, const int32_t* req_indptr,
+                 const int32_t* kv_tbl_indptr, const uint32_t* kv_tbl, const int32_t* prefix_lens,
+                 int n_req, int n_tokens, int n_kv_heads, fl_stream stream);
+
+/* ---------------------------------------------------------------- paged attention (Section 2.1, Section 4.2)
+ * For request i, query head h (KV head h / (n_q_heads / n_kv_heads)) and new token j:
+ *     out = softmax_{u <= prefix_lens[i] + j}(sm_scale * <q, k_u>) . v_u
+ * over the request's keys/values read from pool blocks through its table: the cached prefix is
+ * reused as stored, the new tokens (already appended) are causal.  Prefill, decode (new_len 1) and
+ * mixed batches go through the same call.  q, out: device [n_tokens, n_q_heads, 128] bf16 packed by
+ * request (req_indptr); new_lens[i] = req_indptr[i+1] - req_indptr[i].  n_tbl = total number of
+ * table entries.  Needs block tokens bt = 16.  workspace: device scratch of at least
+ * fl_paged_attention_workspace(...) bytes; same sharing rule as above. */
+size_t fl_paged_attention_workspace(int n_req, int n_tokens, int n_tbl, int n_q_heads, int n_kv_heads);
+int fl_paged_attention(fl_pool* pool, fl_bf16* out, const fl_bf16* q, const int32_t* req_indptr,
+                       const int32_t* kv_tbl_indptr, const uint32_t* kv_tbl, const int32_t* prefix_lens,
+                       const int32_t* new_lens, int n_req, int n_tokens, int n_tbl,
+                       int n_q_heads, int n_kv_heads, float sm_scale,
+                       void* workspace, size_t workspace_bytes, fl_stream stream);
+
+/* ---------------------------------------------------------------- swap (Section 4.3 "Asynchronous Swapping-in/out")
+ * Copies whole blocks between the device slab and the pinned host slab, pair k = (dev_ids[k],
+ * host_ids[k]) (host pointers), in list order, asynchronously on `side` (copy engines), so that it
+ * overlaps kernels running on other streams.  Every listed block must be allocated (FL_EBADID,
+ * nothing copied).  The caller guarantees that no kernel in flight touches the listed device blocks
+ * (the paper evicts only nodes no running query uses, and a query whose blocks are in flight waits).
+ * fl_swap_record records `ev` on the side stream; fl_swap_wait polls it on the host until done or
+ * timeout_ms elapsed (FL_ETIMEOUT) - no device-side waiting. */
+int fl_swap_out(fl_pool* pool, const uint32_t* dev_ids, const uint32_t* host_ids, uint32_t n, fl_stream side);
+int fl_swap_in(fl_pool* pool, const uint32_t* dev_ids, const uint32_t* host_ids, uint32_t n, fl_stream side);
+int fl_swap_record(fl_pool* pool, fl_event ev, fl_stream side);
+int fl_swap_wait(fl_pool* pool, fl_event ev, int timeout_ms);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FASTPOOL_H */

@@ -1,0 +1,283 @@
+"""ctypes binding of libfastpool.so: argument marshalling only, one Python function per C call,
+same names.  Device arguments are torch CUDA tensors (or raw integer addresses), host id lists are
+numpy arrays.  Every step of the path runs inside the library; there is no Python or CPU fallback:
+if the library has not been built, importing this module raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libfastpool.so")
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2505_03756_b200.build` "
+                      "(there is no fallback path)")
+lib = C.CDLL(LIB_PATH)
+
+FL_OK, FL_EINVAL, FL_ENOMEM, FL_EBADID, FL_EBUSY, FL_ECUDA, FL_ETIMEOUT = 0, -1, -2, -3, -4, -5, -6
+_NAMES = {0: "FL_OK", -1: "FL_EINVAL", -2: "FL_ENOMEM", -3: "FL_EBADID", -4: "FL_EBUSY", -5: "FL_ECUDA",
+          -6: "FL_ETIMEOUT"}
+
+
+class FlError(RuntimeError):
+    def __init__(self, code, where):
+        super().__init__(f"{where}: {_NAMES.get(code, code)}")
+        self.code = code
+
+
+class fl_lora_shape(C.Structure):
+    _fields_ = [("d_in", C.c_int32), ("d_out", C.c_int32)]
+
+
+class fl_status(C.Structure):
+    _fields_ = [("device_flags", C.c_uint32), ("blocks_used", C.c_uint32), ("blocks_free", C.c_uint32),
+                ("host_blocks_used", C.c_uint32), ("host_blocks_free", C.c_uint32), ("lora_blocks", C.c_uint32),
+                ("bytes_swapped_in", C.c_uint64), ("bytes_swapped_out", C.c_uint64)]
+
+
+_vp, _u32p, _i32p = C.c_void_p, C.POINTER(C.c_uint32), C.POINTER(C.c_int32)
+_SIGS = {
+    "fl_pool_create": (C.c_int, [C.POINTER(_vp), C.c_size_t, C.c_uint32, C.c_uint32, C.c_int]),
+    "fl_pool_destroy": (C.c_int, [_vp]),
+    "fl_block_alloc": (C.c_int, [_vp, C.c_uint32, _vp]),
+    "fl_block_free": (C.c_int, [_vp, C.c_uint32, _vp]),
+    "fl_host_block_alloc": (C.c_int, [_vp, C.c_uint32, _vp]),
+    "fl_host_block_free": (C.c_int, [_vp, C.c_uint32, _vp]),
+    "fl_pool_device_base": (_vp, [_vp]),
+    "fl_pool_host_base": (_vp, [_vp]),
+    "fl_block_read": (C.c_int, [_vp, C.c_uint32, _vp]),
+    "fl_block_write": (C.c_int, [_vp, C.c_uint32, _vp]),
+    "fl_pool_snapshot": (C.c_int, [_vp, C.c_int, _vp, C.c_uint32, _u32p]),
+    "fl_pool_status": (C.c_int, [_vp, C.POINTER(fl_status), C.c_int]),
+    "fl_last_cuda_error": (C.c_int, [_vp]),
+    "fl_lora_blocks": (C.c_int, [C.c_size_t, C.c_int32, C.POINTER(fl_lora_shape), C.c_int, _u32p]),
+    "fl_lora_pack_host": (C.c_int, [_vp, C.c_int32, C.POINTER(fl_lora_shape), C.c_int, C.POINTER(_vp),
+                                    C.POINTER(_vp), _vp, C.c_uint32]),
+    "fl_lora_register": (C.c_int, [_vp, C.c_int32, C.c_int32, C.POINTER(fl_lora_shape), C.c_int, _vp, C.c_uint32]),
+    "fl_lora_unregister": (C.c_int, [_vp, C.c_int32]),
+    "fl_lora_sgmv_workspace": (C.c_size_t, [C.c_int, C.c_int]),
+    "fl_lora_sgmv": (C.c_int, [_vp, _vp, _vp, C.c_int, _vp, _vp, C.c_int, C.c_int, C.c_float, _vp, C.c_size_t, _vp]),
+    "fl_lora_sgmv_multi": (C.c_int, [_vp, C.POINTER(_vp), _vp, _i32p, C.c_int, _vp, _vp, C.c_int, C.c_int,
+                                     C.c_float, _vp, C.c_size_t, _vp]),
+    "fl_kv_append": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, C.c_int, C.c_int, C.c_int, _vp]),
+    "fl_paged_attention_workspace": (C.c_size_t, [C.c_int, C.c_int, C.c_int, C.c_int, C.c_int]),
+    "fl_paged_attention": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, C.c_int, C.c_int, C.c_int, C.c_int,
+                                     C.c_int, C.c_float, _vp, C.c_size_t, _vp]),
+    "fl_swap_out": (C.c_int, [_vp, _vp, _vp, C.c_uint32, _vp]),
+    "fl_swap_in": (C.c_int, [_vp, _vp, _vp, C.c_uint32, _vp]),
+    "fl_swap_record": (C.c_int, [_vp, _vp, _vp]),
+    "fl_swap_wait": (C.c_int, [_vp, _vp, C.c_int]),
+}
+for _n, (_r, _a) in _SIGS.items():
+    getattr(lib, _n).restype = _r
+    getattr(lib, _n).argtypes = _a
+EXPORTS = tuple(_SIGS)
+
+
+def _check(code, where):
+    if code != FL_OK:
+        raise FlError(code, where)
+
+
+def _dev(t):
+    """Device address of a torch tensor (or pass an int / None through)."""
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return t
+    assert t.is_cuda and t.is_contiguous()
+    return t.data_ptr()
+
+
+def _ids(a):
+    a = np.ascontiguousarray(a, dtype=np.uint32)
+    return a, a.ctypes.data
+
+
+def _stream(s):
+    if s is None:
+        import torch
+        return torch.cuda.current_stream().cuda_stream
+    return s if isinstance(s, int) else s.cuda_stream
+
+
+def _shapes(mats):
+    arr = (fl_lora_shape * len(mats))()
+    for i, (d_in, d_out) in enumerate(mats):
+        arr[i].d_in, arr[i].d_out = int(d_in), int(d_out)
+    return arr
+
+
+# ------------------------------------------------------------------ one function per C call
+def fl_pool_create(block_bytes, n_blocks, n_host_blocks, device=0):
+    h = _vp()
+    _check(lib.fl_pool_create(C.byref(h), block_bytes, n_blocks, n_host_blocks, device), "fl_pool_create")
+    return h
+
+
+def fl_pool_destroy(pool):
+    _check(lib.fl_pool_destroy(pool), "fl_pool_destroy")
+
+
+def _alloc(fn, name, pool, n):
+    ids = np.empty(n, dtype=np.uint32)
+    _check(fn(pool, n, ids.ctypes.data), name)
+    return ids
+
+
+def fl_block_alloc(pool, n):
+    return _alloc(lib.fl_block_alloc, "fl_block_alloc", pool, n)
+
+
+def fl_host_block_alloc(pool, n):
+    return _alloc(lib.fl_host_block_alloc, "fl_host_block_alloc", pool, n)
+
+
+def fl_block_free(pool, ids):
+    a, p = _ids(ids)
+    _check(lib.fl_block_free(pool, len(a), p), "fl_block_free")
+
+
+def fl_host_block_free(pool, ids):
+    a, p = _ids(ids)
+    _check(lib.fl_host_block_free(pool, len(a), p), "fl_host_block_free")
+
+
+def fl_pool_device_base(pool):
+    return lib.fl_pool_device_base(pool)
+
+
+def fl_pool_host_base(pool):
+    return lib.fl_pool_host_base(pool)
+
+
+def fl_block_read(pool, block_id, block_bytes):
+    out = np.empty(block_bytes, dtype=np.uint8)
+    _check(lib.fl_block_read(pool, int(block_id), out.ctypes.data), "fl_block_read")
+    return out
+
+
+def fl_block_write(pool, block_id, data):
+    data = np.ascontiguousarray(data, dtype=np.uint8)
+    _check(lib.fl_block_write(pool, int(block_id), data.ctypes.data), "fl_block_write")
+
+
+def fl_pool_snapshot(pool, host=False):
+    n = C.c_uint32()
+    _check(lib.fl_pool_snapshot(pool, int(host), None, 0, C.byref(n)), "fl_pool_snapshot")
+    ids = np.empty(n.value, dtype=np.uint32)
+    _check(lib.fl_pool_snapshot(pool, int(host), ids.ctypes.data, n.value, C.byref(n)), "fl_pool_snapshot")
+    return ids
+
+
+def fl_pool_status(pool, clear=False):
+    st = fl_status()
+    _check(lib.fl_pool_status(pool, C.byref(st), int(clear)), "fl_pool_status")
+    return {k: getattr(st, k) for k, _ in fl_status._fields_}
+
+
+def fl_last_cuda_error(pool):
+    return lib.fl_last_cuda_error(pool)
+
+
+def fl_lora_blocks(block_bytes, rank, mats):
+    n = C.c_uint32()
+    _check(lib.fl_lora_blocks(block_bytes, rank, _shapes(mats), len(mats), C.byref(n)), "fl_lora_blocks")
+    return n.value
+
+
+def fl_lora_pack_host(pool, rank, mats, A_bits, B_bits, host_blocks):
+    """A_bits[m]: numpy uint16 [d_in, rank]; B_bits[m]: numpy uint16 [rank, d_out] (bf16 bit patterns)."""
+    A = [np.ascontiguousarray(a, dtype=np.uint16) for a in A_bits]
+    B = [np.ascontiguousarray(b, dtype=np.uint16) for b in B_bits]
+    pa = (_vp * len(A))(*[a.ctypes.data for a in A])
+    pb = (_vp * len(B))(*[b.ctypes.data for b in B])
+    ids, p = _ids(host_blocks)
+    _check(lib.fl_lora_pack_host(pool, rank, _shapes(mats), len(mats), pa, pb, p, len(ids)), "fl_lora_pack_host")
+
+
+def fl_lora_register(pool, lora_id, rank, mats, block_table):
+    ids, p = _ids(block_table)
+    _check(lib.fl_lora_register(pool, lora_id, rank, _shapes(mats), len(mats), p, len(ids)), "fl_lora_register")
+
+
+def fl_lora_unregister(pool, lora_id):
+    _check(lib.fl_lora_unregister(pool, lora_id), "fl_lora_unregister")
+
+
+def fl_lora_sgmv_workspace(n_tokens, n_mats=1):
+    return lib.fl_lora_sgmv_workspace(n_tokens, n_mats)
+
+
+def fl_lora_sgmv(pool, y, x, mat_index, seg_indptr, lora_ids, n_seg, n_tokens, scale, workspace, stream=None):
+    _check(lib.fl_lora_sgmv(pool, _dev(y), _dev(x), mat_index, _dev(seg_indptr), _dev(lora_ids), n_seg, n_tokens,
+                            scale, _dev(workspace), workspace.numel() * workspace.element_size(), _stream(stream)),
+           "fl_lora_sgmv")
+
+
+def fl_lora_sgmv_multi(pool, ys, x, mat_indices, seg_indptr, lora_ids, n_seg, n_tokens, scale, workspace, stream=None):
+    py = (_vp * len(ys))(*[_dev(y) for y in ys])
+    mi = (C.c_int32 * len(ys))(*[int(m) for m in mat_indices])
+    _check(lib.fl_lora_sgmv_multi(pool, py, _dev(x), mi, len(ys), _dev(seg_indptr), _dev(lora_ids), n_seg, n_tokens,
+                                  scale, _dev(workspace), workspace.numel() * workspace.element_size(),
+                                  _stream(stream)), "fl_lora_sgmv_multi")
+
+
+def fl_kv_append(pool, k_new, v_new, req_indptr, kv_tbl_indptr, kv_tbl, prefix_lens, n_req, n_tokens, n_kv_heads,
+                 stream=None):
+    _check(lib.fl_kv_append(pool, _dev(k_new), _dev(v_new), _dev(req_indptr), _dev(kv_tbl_indptr), _dev(kv_tbl),
+                            _dev(prefix_lens), n_req, n_tokens, n_kv_heads, _stream(stream)), "fl_kv_append")
+
+
+def fl_paged_attention_workspace(n_req, n_tokens, n_tbl, n_q_heads, n_kv_heads):
+    return lib.fl_paged_attention_workspace(n_req, n_tokens, n_tbl, n_q_heads, n_kv_heads)
+
+
+def fl_paged_attention(pool, out, q, req_indptr, kv_tbl_indptr, kv_tbl, prefix_lens, new_lens, n_req, n_tokens, n_tbl,
+                       n_q_heads, n_kv_heads, sm_scale, workspace, stream=None):
+    _check(lib.fl_paged_attention(pool, _dev(out), _dev(q), _dev(req_indptr), _dev(kv_tbl_indptr), _dev(kv_tbl),
+                                  _dev(prefix_lens), _dev(new_lens), n_req, n_tokens, n_tbl, n_q_heads, n_kv_heads,
+                                  sm_scale, _dev(workspace), workspace.numel() * workspace.element_size(),
+                                  _stream(stream)), "fl_paged_attention")
+
+
+def fl_swap_out(pool, dev_ids, host_ids, side_stream):
+    d, pd = _ids(dev_ids)
+    h, ph = _ids(host_ids)
+    assert len(d) == len(h)
+    _check(lib.fl_swap_out(pool, pd, ph, len(d), _stream(side_stream)), "fl_swap_out")
+
+
+def fl_swap_in(pool, dev_ids, host_ids, side_stream):
+    d, pd = _ids(dev_ids)
+    h, ph = _ids(host_ids)
+    assert len(d) == len(h)
+    _check(lib.fl_swap_in(pool, pd, ph, len(d), _stream(side_stream)), "fl_swap_in")
+
+
+def fl_swap_record(pool, event, side_stream):
+    _check(lib.fl_swap_record(pool, event.cuda_event, _stream(side_stream)), "fl_swap_record")
+
+
+def fl_swap_wait(pool, event, timeout_ms):
+    return lib.fl_swap_wait(pool, event.cuda_event, timeout_ms)
+
+
+# ------------------------------------------------------------------ views of the two slabs (for tests and tools)
+def device_block_bytes(pool, block_bytes, ids):
+    """Copies the listed device blocks to host: uint8 [len(ids), block_bytes]."""
+    out = np.empty((len(ids), block_bytes), dtype=np.uint8)
+    for k, b in enumerate(ids):
+        out[k] = fl_block_read(pool, b, block_bytes)
+    return out
+
+
+def host_slab(pool, block_bytes, n_host_blocks):
+    """numpy uint8 view [n_host_blocks, block_bytes] of the pinned host slab."""
+    base = fl_pool_host_base(pool)
+    buf = (C.c_uint8 * (block_bytes * n_host_blocks)).from_address(base)
+    return np.frombuffer(buf, dtype=np.uint8).reshape(n_host_blocks, block_bytes)

@@ -1,0 +1,85 @@
+// Internal definitions shared by the translation units of libfastpool.
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <map>
+#include <vector>
+#include "fastpool.h"
+
+// Placement of one projection's rank-row streams inside its adapter's block table.
+struct LoraMat {
+  uint32_t a_tab, a_row0, a_rpb;   // table entry of the class, first row inside the class, rows per block
+  uint32_t b_tab, b_row0, b_rpb;
+  int32_t d_in, d_out;
+};
+// Device-side adapter directory entry, indexed by lora id.
+struct LoraEntry {
+  int32_t rank;        // 0 = not registered
+  int32_t n_mats;
+  uint32_t table_off;  // first entry of this adapter's table inside the table arena
+  uint32_t n_table;
+  LoraMat mats[FL_MAX_MATS];
+};
+
+// What kernels need to address the pool.
+struct PoolView {
+  unsigned char* slab;
+  size_t block_bytes;
+  uint32_t n_blocks;
+  const LoraEntry* dir;
+  uint32_t dir_cap;
+  const uint32_t* tables;
+  uint32_t* flags;     // sticky status word
+};
+
+enum { FLAG_BAD_BLOCK = 1, FLAG_BAD_POS = 2, FLAG_BAD_LORA = 4, FLAG_WAIT_GAVE_UP = 8 };
+
+struct BlockStack {
+  std::vector<uint32_t> free;   // top = back
+  std::vector<uint8_t> used;
+  void init(uint32_t n) {
+    free.resize(n);
+    for (uint32_t i = 0; i < n; ++i) free[i] = n - 1 - i;
+    used.assign(n, 0);
+  }
+};
+
+struct fl_pool {
+  int device = 0;
+  size_t block_bytes = 0;
+  uint32_t n_blocks = 0, n_host_blocks = 0;
+  unsigned char* slab = nullptr;
+  unsigned char* host_slab = nullptr;
+  BlockStack dev, host;
+  // adapter directory
+  LoraEntry* d_dir = nullptr;
+  uint32_t dir_cap = 0;
+  uint32_t* d_tables = nullptr;
+  uint32_t tables_cap = 0;
+  std::map<uint32_t, uint32_t> arena_free;        // offset -> length of free table-arena ranges
+  std::map<int32_t, LoraEntry> registered;        // host mirror
+  int n_mats = 0;
+  fl_lora_shape mats[FL_MAX_MATS];
+  int max_rank = 0;
+  uint32_t lora_blocks = 0;
+  uint32_t* d_flags = nullptr;
+  uint64_t bytes_in = 0, bytes_out = 0;
+  int last_cuda = 0;
+  int sm_count = 148;
+  void* tmap_cache = nullptr;                      // tensor maps of the slab, keyed by KV head count
+  PoolView view() const { return PoolView{slab, block_bytes, n_blocks, d_dir, dir_cap, d_tables, d_flags}; }
+};
+
+#define FL_CUDA(pool, call)                                  \
+  do {                                                       \
+    cudaError_t e__ = (call);                                \
+    if (e__ != cudaSuccess) {                                \
+      if (pool) (pool)->last_cuda = (int)e__;                \
+      return FL_ECUDA;                                       \
+    }                                                        \
+  } while (0)
+
+// Layout arithmetic of an adapter (host side).
+int fl_layout_adapter(size_t block_bytes, int32_t rank, const fl_lora_shape* mats, int n_mats,
+                      LoraMat* out, uint32_t* n_table);

@@ -1,0 +1,440 @@
+// Segmented LoRA projection y += scale * (x A_i) B_i over adapter rank-rows stored in pool blocks
+// (Eq. 1, Eq. 2; the segmented batching of Section 2.1).
+//
+// Two kernels.  shrink: v = x A_i for a tile of tokens of one segment and a slice of d_in, adapter
+// rows fetched through the adapter's block table with 16-byte cp.async, bf16 mma.sync with fp32
+// accumulation, partial sums written to scratch [mat][k-slice][token][RMAX].  expand: sums the
+// partials, scales, splits v into bf16 hi + lo parts (so the second contraction keeps fp32-level
+// accuracy), multiplies by the B rows of a column range and adds into y with coalesced 16-byte
+// read-modify-write staged through shared memory.  Both are bound by HBM traffic (x and y rows
+// for long segments, adapter rows for decode-sized segments), not by the contraction.
+#include "mma_utils.cuh"
+#include "pool.cuh"
+
+namespace {
+
+constexpr int SG_THREADS = 128;
+constexpr int KS = 64;            // d_in elements per shrink pipeline stage (128-byte rows)
+constexpr int SH_STAGES = 4;
+constexpr int NSUB = 128;         // y columns per expand sub-tile (256-byte rows)
+constexpr int EXPAND_COLS = 512;  // y columns per expand CTA
+constexpr int KSPLIT_MAX = 8;
+
+struct SgmvArgs {
+  PoolView pv;
+  const __nv_bfloat16* x;
+  __nv_bfloat16* y[FL_MAX_MATS];
+  int mat_index[FL_MAX_MATS];
+  int n_mats;
+  const int32_t* seg_indptr;
+  const int32_t* lora_ids;
+  int n_seg, n_tokens;
+  float scale;
+  float* v;        // [n_mats][ksplit][n_tokens][RMAX]
+  int ksplit;
+};
+
+// Token tile `tile` (tiles of TM tokens, counted over segments that carry an adapter) -> segment and
+// token range.  Every warp evaluates it redundantly with a warp scan over 32 segments at a time.
+template <int TM>
+__device__ __forceinline__ bool find_tile(const int32_t* __restrict__ seg_indptr, const int32_t* __restrict__ lora_ids,
+                                          int n_seg, int tile, int& seg, int& tok0, int& tok1) {
+  const int lane = threadIdx.x & 31;
+  int base = 0;
+  for (int s0 = 0; s0 < n_seg; s0 += 32) {
+    const int s = s0 + lane;
+    int lo = 0, hi = 0, nt = 0;
+    if (s < n_seg) {
+      lo = seg_indptr[s];
+      hi = seg_indptr[s + 1];
+      if (lora_ids[s] >= 0 && hi > lo) nt = (hi - lo + TM - 1) / TM;
+    }
+    int incl = nt;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      const int o = __shfl_up_sync(0xffffffffu, incl, d);
+      if (lane >= d) incl += o;
+    }
+    const int total = __shfl_sync(0xffffffffu, incl, 31);
+    if (tile < base + total) {
+      const int first = base + incl - nt;
+      const bool mine = nt > 0 && tile >= first && tile < first + nt;
+      const int src = __ffs(__ballot_sync(0xffffffffu, mine)) - 1;
+      const int k = tile - __shfl_sync(0xffffffffu, first, src);
+      seg = s0 + src;
+      tok0 = __shfl_sync(0xffffffffu, lo, src) + k * TM;
+      tok1 = min(tok0 + TM, __shfl_sync(0xffffffffu, hi, src));
+      return true;
+    }
+    base += total;
+  }
+  return false;
+}
+
+// Start of rank-row `row` of a stream (class table entry tab, first row row0, rows per block rpb, row width).
+__device__ __forceinline__ const unsigned char* lora_row(const PoolView& pv, uint32_t table_off, uint32_t tab,
+                                                         uint32_t row0, uint32_t rpb, int width, int row, bool& ok) {
+  const uint32_t g = row0 + (uint32_t)row;
+  const uint32_t blk = pv.tables[table_off + tab + g / rpb];
+  if (blk >= pv.n_blocks) {
+    atomicOr(pv.flags, (uint32_t)FLAG_BAD_BLOCK);
+    ok = false;
+    return pv.slab;
+  }
+  ok = true;
+  return pv.slab + (size_t)blk * pv.block_bytes + (size_t)(g % rpb) * 2 * (size_t)width;
+}
+
+template <int TM, int RMAX>
+__global__ void __launch_bounds__(SG_THREADS) sgmv_shrink_kernel(const SgmvArgs a) {
+  extern __shared__ __align__(128) unsigned char smem[];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int j = blockIdx.x % a.n_mats;
+  const int tile = blockIdx.x / a.n_mats;
+  const int split = blockIdx.y;
+  int seg, tok0, tok1;
+  if (!find_tile<TM>(a.seg_indptr, a.lora_ids, a.n_seg, tile, seg, tok0, tok1)) return;
+  const int lid = a.lora_ids[seg];
+  if ((uint32_t)lid >= a.pv.dir_cap || a.pv.dir[lid].rank <= 0 || a.mat_index[j] >= a.pv.dir[lid].n_mats) {
+    if (tid == 0) atomicOr(a.pv.flags, (uint32_t)FLAG_BAD_LORA);
+    return;
+  }
+  const LoraEntry* e = a.pv.dir + lid;
+  const LoraMat lm = e->mats[a.mat_index[j]];
+  const int rank = min(e->rank, RMAX);
+  const uint32_t table_off = e->table_off;
+  const int d_in = lm.d_in;
+  const int kchunk = ((d_in + a.ksplit * KS - 1) / (a.ksplit * KS)) * KS;
+  const int kb = split * kchunk, ke = min(d_in, kb + kchunk);
+  const int n_it = ke > kb ? (ke - kb + KS - 1) / KS : 0;
+
+  constexpr int XR = TM / 16;      // x rows per thread per stage
+  constexpr int AR = RMAX / 16;    // adapter rows per thread per stage
+  constexpr int STAGE_BYTES = (TM + RMAX) * 128;
+  const int crow = tid >> 3, cchunk = tid & 7;
+  const __nv_bfloat16* xrow[XR];
+  bool xok[XR];
+#pragma unroll
+  for (int i = 0; i < XR; ++i) {
+    const int t = tok0 + crow + 16 * i;
+    xok[i] = t < tok1;
+    xrow[i] = a.x + (size_t)(xok[i] ? t : tok0) * d_in;
+  }
+  const __nv_bfloat16* arow[AR];
+  bool aok[AR];
+#pragma unroll
+  for (int i = 0; i < AR; ++i) {
+    const int r = crow + 16 * i;
+    aok[i] = false;
+    arow[i] = reinterpret_cast<const __nv_bfloat16*>(a.pv.slab);
+    if (r < rank)
+      arow[i] = reinterpret_cast<const __nv_bfloat16*>(
+          lora_row(a.pv, table_off, lm.a_tab, lm.a_row0, lm.a_rpb, d_in, r, aok[i]));
+  }
+  const uint32_t sbase = smem_u32(smem);
+  auto load_stage = [&](int it, int st) {
+    const int kk = kb + it * KS + cchunk * 8;
+    const bool kok = kk < ke;
+    const uint32_t xs = sbase + st * STAGE_BYTES, as = xs + TM * 128;
+#pragma unroll
+    for (int i = 0; i < XR; ++i) cp_async16(xs + swz(crow + 16 * i, cchunk, 8), xrow[i] + kk, xok[i] && kok);
+#pragma unroll
+    for (int i = 0; i < AR; ++i) cp_async16(as + swz(crow + 16 * i, cchunk, 8), arow[i] + kk, aok[i] && kok);
+  };
+
+  float acc[RMAX / 8][4];
+#pragma unroll
+  for (int n = 0; n < RMAX / 8; ++n) acc[n][0] = acc[n][1] = acc[n][2] = acc[n][3] = 0.f;
+
+#pragma unroll
+  for (int s = 0; s < SH_STAGES - 1; ++s) {
+    if (s < n_it) load_stage(s, s);
+    cp_async_commit();
+  }
+  const int mrow = (TM == 64 ? warp * 16 : 0) + (lane & 7) + 8 * ((lane >> 3) & 1);
+  for (int it = 0; it < n_it; ++it) {
+    cp_async_wait<SH_STAGES - 2>();
+    __syncthreads();
+    if (it + SH_STAGES - 1 < n_it) load_stage(it + SH_STAGES - 1, (it + SH_STAGES - 1) % SH_STAGES);
+    cp_async_commit();
+    const uint32_t xs = sbase + (it % SH_STAGES) * STAGE_BYTES, as = xs + TM * 128;
+#pragma unroll
+    for (int ks = 0; ks < KS / 16; ++ks) {
+      if (TM == 16 && ks != warp) continue;   // short tiles: the four warps split each stage along k
+      uint32_t af[4];
+      ldmatrix_x4(af, xs + swz(mrow, 2 * ks + (lane >> 4), 8));
+#pragma unroll
+      for (int p = 0; p < RMAX / 16; ++p) {
+        if (16 * p < rank) {
+          uint32_t bf[4];
+          ldmatrix_x4(bf, as + swz(16 * p + (lane & 7) + 8 * (lane >> 4), 2 * ks + ((lane >> 3) & 1), 8));
+          mma_bf16(acc[2 * p], af, bf[0], bf[1]);
+          mma_bf16(acc[2 * p + 1], af, bf[2], bf[3]);
+        }
+      }
+    }
+  }
+  float* vout = a.v + ((size_t)(j * a.ksplit + split) * a.n_tokens) * RMAX;
+  const int g = lane >> 2, t4 = lane & 3;
+  if (TM == 64) {
+#pragma unroll
+    for (int n = 0; n < RMAX / 8; ++n) {
+      const int r0 = tok0 + warp * 16 + g;
+      if (r0 < tok1) *reinterpret_cast<float2*>(vout + (size_t)r0 * RMAX + 8 * n + 2 * t4) = make_float2(acc[n][0], acc[n][1]);
+      if (r0 + 8 < tok1) *reinterpret_cast<float2*>(vout + (size_t)(r0 + 8) * RMAX + 8 * n + 2 * t4) = make_float2(acc[n][2], acc[n][3]);
+    }
+  } else {
+    cp_async_wait<0>();
+    __syncthreads();
+    float* red = reinterpret_cast<float*>(smem);   // [4 warps][16 rows][RMAX]
+#pragma unroll
+    for (int n = 0; n < RMAX / 8; ++n) {
+      float* r = red + (warp * 16 + g) * RMAX + 8 * n + 2 * t4;
+      r[0] = acc[n][0]; r[1] = acc[n][1];
+      r[8 * RMAX] = acc[n][2]; r[8 * RMAX + 1] = acc[n][3];
+    }
+    __syncthreads();
+    for (int i = tid; i < 16 * RMAX; i += SG_THREADS) {
+      const int row = i / RMAX;
+      if (tok0 + row < tok1)
+        vout[(size_t)(tok0 + row) * RMAX + (i % RMAX)] =
+            red[i] + red[16 * RMAX + i] + red[32 * RMAX + i] + red[48 * RMAX + i];
+    }
+  }
+}
+
+template <int TM, int RMAX>
+__global__ void __launch_bounds__(SG_THREADS) sgmv_expand_kernel(const SgmvArgs a) {
+  extern __shared__ __align__(128) unsigned char smem[];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int j = blockIdx.x % a.n_mats;
+  const int tile = blockIdx.x / a.n_mats;
+  int seg, tok0, tok1;
+  if (!find_tile<TM>(a.seg_indptr, a.lora_ids, a.n_seg, tile, seg, tok0, tok1)) return;
+  const int lid = a.lora_ids[seg];
+  if ((uint32_t)lid >= a.pv.dir_cap || a.pv.dir[lid].rank <= 0 || a.mat_index[j] >= a.pv.dir[lid].n_mats) return;
+  const LoraEntry* e = a.pv.dir + lid;
+  const LoraMat lm = e->mats[a.mat_index[j]];
+  const int rank = min(e->rank, RMAX);
+  const uint32_t table_off = e->table_off;
+  const int d_out = lm.d_out;
+  const int c0 = blockIdx.y * EXPAND_COLS;
+  if (c0 >= d_out) return;
+  const int c1 = min(d_out, c0 + EXPAND_COLS);
+  const int n_sub = (c1 - c0 + NSUB - 1) / NSUB;
+
+  constexpr int WM = TM / 16, WN = 4 / WM;     // warps along tokens / along columns
+  constexpr int NTW = 16 / WN;                 // 8-column tiles per warp inside a sub-tile
+  const int warp_m = warp % WM, warp_n = warp / WM;
+  const int g = lane >> 2, t4 = lane & 3;
+
+  // v fragments: sum of the k-slices, scaled, as bf16 hi + lo
+  uint32_t ahi[RMAX / 16][4], alo[RMAX / 16][4];
+  {
+    const int r0 = tok0 + warp_m * 16 + g, r1 = r0 + 8;
+#pragma unroll
+    for (int ks = 0; ks < RMAX / 16; ++ks) {
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const int row = (q & 1) ? r1 : r0;
+        const int col = 16 * ks + 2 * t4 + ((q & 2) ? 8 : 0);
+        float2 s = make_float2(0.f, 0.f);
+        if (row < tok1 && col < rank) {
+          for (int sp = 0; sp < a.ksplit; ++sp) {
+            const float2 p = *reinterpret_cast<const float2*>(
+                a.v + ((size_t)(j * a.ksplit + sp) * a.n_tokens + row) * RMAX + col);
+            s.x += p.x; s.y += p.y;
+          }
+        }
+        s.x *= a.scale; s.y *= a.scale;
+        const __nv_bfloat16 hx = __float2bfloat16_rn(s.x), hy = __float2bfloat16_rn(s.y);
+        ahi[ks][q] = pack_bf16(__bfloat162float(hx), __bfloat162float(hy));
+        alo[ks][q] = pack_bf16(s.x - __bfloat162float(hx), s.y - __bfloat162float(hy));
+      }
+    }
+  }
+
+  constexpr int YR = TM / 8;       // y rows per thread per sub-tile
+  constexpr int BR = RMAX / 8;     // adapter rows per thread per sub-tile
+  constexpr int STAGE_BYTES = (TM + RMAX) * 256;
+  const int crow = tid >> 4, cchunk = tid & 15;
+  __nv_bfloat16* yrow[YR];
+  bool yok[YR];
+#pragma unroll
+  for (int i = 0; i < YR; ++i) {
+    const int t = tok0 + crow + 8 * i;
+    yok[i] = t < tok1;
+    yrow[i] = a.y[j] + (size_t)(yok[i] ? t : tok0) * d_out;
+  }
+  const __nv_bfloat16* brow[BR];
+  bool bok[BR];
+#pragma unroll
+  for (int i = 0; i < BR; ++i) {
+    const int r = crow + 8 * i;
+    bok[i] = false;
+    brow[i] = reinterpret_cast<const __nv_bfloat16*>(a.pv.slab);
+    if (r < rank)
+      brow[i] = reinterpret_cast<const __nv_bfloat16*>(
+          lora_row(a.pv, table_off, lm.b_tab, lm.b_row0, lm.b_rpb, d_out, r, bok[i]));
+  }
+  const uint32_t sbase = smem_u32(smem);
+  auto load_sub = [&](int sub, int st) {
+    const int col = c0 + sub * NSUB + cchunk * 8;
+    const bool cok = col < c1;
+    const uint32_t ys = sbase + st * STAGE_BYTES, bs = ys + TM * 256;
+#pragma unroll
+    for (int i = 0; i < YR; ++i) cp_async16(ys + swz(crow + 8 * i, cchunk, 16), yrow[i] + col, yok[i] && cok);
+#pragma unroll
+    for (int i = 0; i < BR; ++i) cp_async16(bs + swz(crow + 8 * i, cchunk, 16), brow[i] + col, bok[i] && cok);
+  };
+
+  load_sub(0, 0);
+  cp_async_commit();
+  for (int sub = 0; sub < n_sub; ++sub) {
+    const int st = sub & 1;
+    if (sub + 1 < n_sub) load_sub(sub + 1, st ^ 1);
+    cp_async_commit();
+    cp_async_wait<1>();
+    __syncthreads();
+    unsigned char* ysm = smem + st * STAGE_BYTES;
+    const uint32_t bs = sbase + st * STAGE_BYTES + TM * 256;
+    float acc[NTW][4];
+#pragma unroll
+    for (int n = 0; n < NTW; ++n) acc[n][0] = acc[n][1] = acc[n][2] = acc[n][3] = 0.f;
+#pragma unroll
+    for (int ks = 0; ks < RMAX / 16; ++ks) {
+      if (16 * ks < rank) {
+#pragma unroll
+        for (int p = 0; p < NTW / 2; ++p) {
+          uint32_t bf[4];
+          ldmatrix_x4_trans(bf, bs + swz(16 * ks + (lane & 7) + 8 * ((lane >> 3) & 1),
+                                         warp_n * NTW + 2 * p + (lane >> 4), 16));
+          mma_bf16(acc[2 * p], ahi[ks], bf[0], bf[1]);
+          mma_bf16(acc[2 * p], alo[ks], bf[0], bf[1]);
+          mma_bf16(acc[2 * p + 1], ahi[ks], bf[2], bf[3]);
+          mma_bf16(acc[2 * p + 1], alo[ks], bf[2], bf[3]);
+        }
+      }
+    }
+    // add into the staged y rows (each element is owned by exactly one thread)
+#pragma unroll
+    for (int n = 0; n < NTW; ++n) {
+      const int chunk = warp_n * NTW + n;
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        const int row = warp_m * 16 + g + 8 * h;
+        uint32_t* p = reinterpret_cast<uint32_t*>(ysm + swz(row, chunk, 16) + 4 * t4);
+        const float2 old = unpack_bf16(*p);
+        *p = pack_bf16(old.x + acc[n][2 * h], old.y + acc[n][2 * h + 1]);
+      }
+    }
+    __syncthreads();
+    {
+      const int col = c0 + sub * NSUB + cchunk * 8;
+      if (col < c1) {
+#pragma unroll
+        for (int i = 0; i < YR; ++i)
+          if (yok[i])
+            *reinterpret_cast<uint4*>(yrow[i] + col) = *reinterpret_cast<const uint4*>(ysm + swz(crow + 8 * i, cchunk, 16));
+      }
+    }
+    __syncthreads();
+  }
+}
+
+int pick_ksplit(int n_tokens) {
+  // decode-sized batches have few token tiles: slice d_in so that enough CTAs stream adapter rows
+  const int tiles = n_tokens / 16 + 1;
+  int ks = 592 / tiles;
+  if (ks < 1) ks = 1;
+  if (ks > KSPLIT_MAX) ks = KSPLIT_MAX;
+  return ks;
+}
+
+template <int TM, int RMAX>
+int launch_pair(fl_pool* p, const SgmvArgs& a, int tiles, int d_out_max, cudaStream_t st) {
+  static bool configured[16] = {};
+  const int shrink_smem = SH_STAGES * (TM + RMAX) * 128;
+  const int expand_smem = 2 * (TM + RMAX) * 256;
+  if (!configured[p->device & 15]) {
+    FL_CUDA(p, cudaFuncSetAttribute(sgmv_shrink_kernel<TM, RMAX>, cudaFuncAttributeMaxDynamicSharedMemorySize, shrink_smem));
+    FL_CUDA(p, cudaFuncSetAttribute(sgmv_expand_kernel<TM, RMAX>, cudaFuncAttributeMaxDynamicSharedMemorySize, expand_smem));
+    configured[p->device & 15] = true;
+  }
+  sgmv_shrink_kernel<TM, RMAX><<<dim3(tiles * a.n_mats, a.ksplit), SG_THREADS, shrink_smem, st>>>(a);
+  sgmv_expand_kernel<TM, RMAX><<<dim3(tiles * a.n_mats, (d_out_max + EXPAND_COLS - 1) / EXPAND_COLS), SG_THREADS, expand_smem, st>>>(a);
+  FL_CUDA(p, cudaGetLastError());
+  return FL_OK;
+}
+
+int rmax_of(const fl_pool* p) { return p->max_rank <= 16 ? 16 : (p->max_rank <= 32 ? 32 : 64); }
+
+}  // namespace
+
+extern "C" {
+
+size_t fl_lora_sgmv_workspace(int n_tokens, int n_mats) {
+  if (n_tokens <= 0 || n_mats <= 0) return 256;
+  return (size_t)n_mats * pick_ksplit(n_tokens) * (size_t)n_tokens * FL_MAX_RANK * sizeof(float) + 256;
+}
+
+int fl_lora_sgmv_multi(fl_pool* p, fl_bf16* const* ys, const fl_bf16* x, const int* mat_indices, int n_mats,
+                       const int32_t* seg_indptr, const int32_t* lora_ids, int n_seg, int n_tokens,
+                       float scale, void* workspace, size_t workspace_bytes, fl_stream stream) {
+  if (!p || n_mats < 1 || n_mats > FL_MAX_MATS || n_seg < 0 || n_tokens < 0 || !ys || !mat_indices) return FL_EINVAL;
+  if (n_seg == 0 || n_tokens == 0) return FL_OK;
+  if (!x || !seg_indptr || !lora_ids || !workspace) return FL_EINVAL;
+  if (p->n_mats == 0) return FL_EBADID;   // no adapter registered
+  SgmvArgs a;
+  a.pv = p->view();
+  a.x = reinterpret_cast<const __nv_bfloat16*>(x);
+  int d_out_max = 0;
+  for (int j = 0; j < n_mats; ++j) {
+    const int mi = mat_indices[j];
+    if (mi < 0 || mi >= p->n_mats || !ys[j]) return FL_EINVAL;
+    if (p->mats[mi].d_in != p->mats[mat_indices[0]].d_in) return FL_EINVAL;   // the projections share x
+    a.y[j] = reinterpret_cast<__nv_bfloat16*>(ys[j]);
+    a.mat_index[j] = mi;
+    d_out_max = d_out_max > p->mats[mi].d_out ? d_out_max : p->mats[mi].d_out;
+  }
+  a.n_mats = n_mats;
+  a.seg_indptr = seg_indptr;
+  a.lora_ids = lora_ids;
+  a.n_seg = n_seg;
+  a.n_tokens = n_tokens;
+  a.scale = scale;
+  a.v = reinterpret_cast<float*>(workspace);
+  a.ksplit = pick_ksplit(n_tokens);
+  if (workspace_bytes < fl_lora_sgmv_workspace(n_tokens, n_mats)) return FL_ENOMEM;
+  int prev = -1;
+  cudaGetDevice(&prev);
+  if (prev != p->device) cudaSetDevice(p->device);
+  const bool small = n_tokens <= 16 * n_seg;   // average segment of at most 16 tokens: decode-like
+  const int rmax = rmax_of(p);
+  const cudaStream_t st = (cudaStream_t)stream;
+  int rc;
+  if (small) {
+    const int tiles = n_seg + n_tokens / 16;
+    rc = rmax == 16 ? launch_pair<16, 16>(p, a, tiles, d_out_max, st)
+       : rmax == 32 ? launch_pair<16, 32>(p, a, tiles, d_out_max, st)
+                    : launch_pair<16, 64>(p, a, tiles, d_out_max, st);
+  } else {
+    const int tiles = n_seg + n_tokens / 64;
+    rc = rmax == 16 ? launch_pair<64, 16>(p, a, tiles, d_out_max, st)
+       : rmax == 32 ? launch_pair<64, 32>(p, a, tiles, d_out_max, st)
+                    : launch_pair<64, 64>(p, a, tiles, d_out_max, st);
+  }
+  if (prev != p->device && prev >= 0) cudaSetDevice(prev);
+  return rc;
+}
+
+int fl_lora_sgmv(fl_pool* p, fl_bf16* y, const fl_bf16* x, int mat_index,
+                 const int32_t* seg_indptr, const int32_t* lora_ids, int n_seg, int n_tokens,
+                 float scale, void* workspace, size_t workspace_bytes, fl_stream stream) {
+  fl_bf16* ys[1] = {y};
+  const int mi[1] = {mat_index};
+  return fl_lora_sgmv_multi(p, ys, x, mi, 1, seg_indptr, lora_ids, n_seg, n_tokens, scale, workspace,
+                            workspace_bytes, stream);
+}
+
+}  // extern "C"

@@ -260,6 +260,8 @@ def fl_swap_in(pool, dev_ids, host_ids, side_stream):
 
 
 def fl_swap_record(pool, event, side_stream):
+    if not event.cuda_event:          # torch creates the CUDA event lazily, on its first record
+        event.record(side_stream if not isinstance(side_stream, int) else None)
     _check(lib.fl_swap_record(pool, event.cuda_event, _stream(side_stream)), "fl_swap_record")
 
 

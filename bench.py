@@ -1,0 +1,382 @@
+#!/usr/bin/env python
+"""Benchmark of the multi-LoRA layer step over the unified block pool.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload prefill7b] [--impl ours|reference]
+
+One step = one pass of the whole hot path over one synthetic batch: block alloc/free for the batch's
+new-token blocks, LoRA q/k/v projection (SGMV), KV append, paged attention over [cached prefix ||
+new tokens], LoRA o projection (plus up/down when the layer has them), and a block swap-out/swap-in
+on a side stream that overlaps the kernels.  Prints one JSON line (rank 0).
+"""
+import argparse
+import json
+import math
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+METRIC = "multi-LoRA layer tokens/s (prefill, decode) on 1 B200; % of HBM/tensor roofline"
+WORKLOAD_TEXT = {
+    "tiny": "configs[0] tiny reference layer",
+    "prefill7b": "configs[1] Llama-2-7B-shaped prefill: 64 requests, 32 adapters rank 16 Zipf(1.0), lengths U{128..1024}, half cached",
+    "decode13b": "configs[2] Llama-2-13B-shaped decode: 256 requests x 1 token, 128 adapters rank 32 Zipf(0.8), contexts U{512..4096}",
+    "gqa34b": "configs[3] 34B-class GQA prefill: 16 requests x (3072 cached + 1024 new), 64q/8kv heads, rank 64, 60 GB pool",
+    "swapstress": "configs[4] swap-stress mixed step: 1000 adapters ranks {8..64}, 64 mixed requests Zipf(1.2), 256 blocks swapped each way per step",
+}
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {"hbm": d["hbm_gbs"], "tensor": d["bf16_tflops"], "tensor_sustained": d.get("bf16_tflops_sustained"),
+                "src": "measured"}
+    return {"hbm": 6650.0, "tensor": 1590.0, "tensor_sustained": 1400.0, "src": "fallback"}
+
+
+# ------------------------------------------------------------------ algorithmic work of each call
+def work_model(wl):
+    s = wl.shape
+    T = wl.n_tokens
+    d = s.head_dim
+    distinct = wl.used_adapters()
+    dims = {n: (i, o) for n, i, o in s.mats}
+
+    def sgmv_bytes(mats):
+        b = 2 * T * dims[mats[0]][0]                                    # x read once
+        for m in mats:
+            b += 4 * T * dims[m][1]                                     # y read + write
+            b += sum(2 * int(wl.ranks[a]) * (dims[m][0] + dims[m][1]) for a in distinct)
+        return b
+
+    n, p = wl.new_lens.astype(np.float64), wl.prefix_lens.astype(np.float64)
+    attn_flops = 4.0 * d * s.n_q_heads * float(np.sum(n * p + n * (n + 1) / 2))
+    attn_bytes = 2 * (2 * T * s.n_q_heads * d) + float(np.sum(p + n)) * 2 * s.n_kv_heads * d * 2
+    w = {
+        "sgmv_qkv": {"bytes": sgmv_bytes(["q", "k", "v"]), "bound": "hbm"},
+        "kv_append": {"bytes": 2 * 2 * T * s.n_kv_heads * d * 2, "bound": "hbm"},
+        "attention": {"bytes": attn_bytes, "flops": attn_flops,
+                      "bound": "tensor" if attn_flops / attn_bytes > 200 else "hbm"},
+        "sgmv_o": {"bytes": sgmv_bytes(["o"]), "bound": "hbm"},
+    }
+    if s.inter:
+        w["sgmv_up"] = {"bytes": sgmv_bytes(["up"]), "bound": "hbm"}
+        w["sgmv_down"] = {"bytes": sgmv_bytes(["down"]), "bound": "hbm"}
+    return w
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons of one GPU through NVML while the timed region runs."""
+
+    def __init__(self, index):
+        super().__init__(daemon=True)
+        self.index, self.samples, self.reasons, self.stop_flag, self.max_mhz = index, [], set(), False, None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def run(self):
+        if self.nv is None:
+            return
+        nv = self.nv
+        names = {nv.nvmlClocksEventReasonSwPowerCap: "sw_power_cap", nv.nvmlClocksEventReasonHwSlowdown: "hw_slowdown",
+                 nv.nvmlClocksEventReasonSwThermalSlowdown: "sw_thermal_slowdown",
+                 nv.nvmlClocksEventReasonHwThermalSlowdown: "hw_thermal_slowdown"}
+        while not self.stop_flag:
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                r = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                for bit, name in names.items():
+                    if r & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(0.01)
+
+    def result(self):
+        self.stop_flag = True
+        if self.nv is None or not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "note": "NVML unavailable"}
+        return {"sm_mhz": float(np.median(self.samples)), "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples)}
+
+
+# ------------------------------------------------------------------ the oracle leg (host cores)
+def oracle_step_sample(wl, n_req_sample):
+    """Runs the oracle's layer step on the first n_req_sample requests of the batch; returns (seconds, tokens)."""
+    from oracle.attention import attend_request
+    from oracle.lora import lora_project
+    s = wl.shape
+    rq = wl.req_indptr
+    T = int(rq[n_req_sample])
+    seg, ids = wl.segments()
+    keep = [k for k in range(len(ids)) if seg[k] < T]
+    seg_s = np.array([min(int(seg[k]), T) for k in keep] + [T], dtype=np.int32)
+    ids_s = ids[keep]
+    x = wl.x("q")[:T]
+    groups = [["q", "k", "v"], ["o"]] + ([["up"], ["down"]] if s.inter else [])
+    yb = {m: wl.y_base(m)[:T] for g in groups for m in g}
+    ad = {m: {a: wl.adapter(a, m) for a in set(int(i) for i in ids_s)} for g in groups for m in g}
+    ctx = [wl.kv_prefix(i) for i in range(n_req_sample)]
+    q = wl.q()[:T]
+    kn, vn = wl.kv_new()
+    xin = {m: (x if m in ("q", "k", "v", "up") else wl.x(m)[:T]) for g in groups for m in g}
+    t0 = time.perf_counter()
+    for g in groups:
+        for m in g:
+            lora_project(yb[m], xin[m], seg_s, ids_s, ad[m], wl.scale)
+    for i in range(n_req_sample):
+        lo, hi = int(rq[i]), int(rq[i + 1])
+        k = np.concatenate([ctx[i][0], kn[lo:hi]])
+        v = np.concatenate([ctx[i][1], vn[lo:hi]])
+        attend_request(q[lo:hi], k, v, int(wl.prefix_lens[i]), 1.0 / math.sqrt(s.head_dim))
+    return time.perf_counter() - t0, T
+
+
+def oracle_baseline(wl, budget_s=12.0):
+    try:
+        from threadpoolctl import threadpool_info
+        cores = max([i.get("num_threads", 1) for i in threadpool_info()] + [1])
+    except Exception:
+        cores = os.cpu_count()
+    n = min(2, wl.n_req)
+    dt, tok = oracle_step_sample(wl, n)
+    per_req = dt / n
+    n2 = int(max(n, min(wl.n_req, budget_s / max(per_req, 1e-6))))
+    if n2 > n:
+        dt, tok = oracle_step_sample(wl, n2)
+        n = n2
+    return {"value": tok / dt, "unit": "tokens/s", "cores": int(cores), "kind": "oracle",
+            "sample": f"first {n} of {wl.n_req} requests ({tok} of {wl.n_tokens} new tokens), whole layer step in "
+                      f"fp64 numpy, {dt:.2f} s"}, dt, tok
+
+
+def run_reference(args, wl):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    vals = []
+    for _ in range(args.warmup + args.steps):
+        cb, dt, tok = oracle_baseline(wl, budget_s=max(1.0, 60.0 / max(1, args.warmup + args.steps)))
+        vals.append((dt, tok, cb))
+    timed = vals[args.warmup:]
+    tot_t = sum(v[0] for v in timed)
+    tot_tok = sum(v[1] for v in timed)
+    value = tot_tok / tot_t
+    cb = dict(timed[-1][2])
+    cb["value"] = value
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * tot_t / len(timed), "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": WORKLOAD_TEXT[args.workload], "note": "CPU oracle on host cores, bounded sample per step"},
+        "cpu_baseline": cb,
+        "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
+
+
+# ------------------------------------------------------------------ the CUDA leg
+def run_ours(args, wl):
+    import torch
+    import torch.distributed as dist
+    from paper_2505_03756_b200 import binding as fl, harness as H, synth
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    if rank > 0:      # requests are independent: every rank runs its own batch of the same shape (no exchange)
+        wl = synth.make_workload(args.workload, seed=wl.seed + 7919 * rank)
+    s = wl.shape
+    T = wl.n_tokens
+    n_swap = args.swap_blocks if args.swap_blocks >= 0 else (256 if args.workload == "swapstress" else 32)
+    sess = H.Session(wl, device=local, extra_host_blocks=2 * n_swap)
+    sess.load_adapters()
+    # the new-token blocks are taken and returned every step (allocator on the path); tables stay put
+    sess.build_batch()
+    sess.fill_prefix_kv()
+    dev = sess.dev
+    groups = [["q", "k", "v"], ["o"]] + ([["up"], ["down"]] if s.inter else [])
+    names = [m for g in groups for m in g]
+    dims = {n: (i, o) for n, i, o in s.mats}
+    # host (pinned) copies of the step's inputs, device buffers
+    h_x = torch.from_numpy(synth.bf16_bits(wl.x("q")).view(np.int16)).pin_memory()
+    h_y = {m: torch.from_numpy(synth.bf16_bits(wl.y_base(m)).view(np.int16)).pin_memory() for m in names}
+    d_x = h_x.to(dev).view(torch.bfloat16)
+    d_y = {m: h_y[m].to(dev).view(torch.bfloat16) for m in names}
+    d_attn = torch.empty(T, s.n_q_heads, s.head_dim, dtype=torch.bfloat16, device=dev)
+    h_out = torch.empty(T, s.hidden, dtype=torch.int16).pin_memory()
+    # swap sets: victims and targets disjoint from the batch's blocks
+    swap_dev_out = sess.alloc(n_swap) if n_swap else np.zeros(0, np.uint32)
+    swap_dev_in = sess.alloc(n_swap) if n_swap else np.zeros(0, np.uint32)
+    swap_host_out = sess.alloc(n_swap, host=True) if n_swap else np.zeros(0, np.uint32)
+    swap_host_in = sess.alloc(n_swap, host=True) if n_swap else np.zeros(0, np.uint32)
+    spare = int(np.sum((wl.new_lens + s.block_tokens - 1) // s.block_tokens))
+    spare = min(spare, fl.fl_pool_status(sess.pool)["blocks_free"])
+    main = torch.cuda.Stream()
+    side = torch.cuda.Stream()
+    ev_side = torch.cuda.Event()
+    calls = ["sgmv_qkv", "kv_append", "attention", "sgmv_o"] + (["sgmv_up", "sgmv_down"] if s.inter else [])
+    launches_per_step = 2 + 1 + 4 + 2 + (4 if s.inter else 0)
+
+    def step(k, evs=None):
+        sign = wl.scale if k % 2 == 0 else -wl.scale     # y += s*delta, then y -= s*delta: values stay bounded
+        ids = fl.fl_block_alloc(sess.pool, spare)        # a1: the allocator runs every step
+        fl.fl_block_free(sess.pool, ids[::-1])
+        if n_swap:                                        # a7: side stream, overlapped
+            fl.fl_swap_out(sess.pool, swap_dev_out, swap_host_out, side)
+            fl.fl_swap_in(sess.pool, swap_dev_in, swap_host_in, side)
+        mark = (lambda: None) if evs is None else (lambda: evs.append(_rec(torch, main)))
+        mark()
+        sess.sgmv([d_y["q"], d_y["k"], d_y["v"]], d_x, ["q", "k", "v"], scale=sign, stream=main)
+        mark()
+        sess.kv_append(d_y["k"], d_y["v"], stream=main)
+        mark()
+        sess.attention(d_attn, d_y["q"], stream=main)
+        mark()
+        sess.sgmv([d_y["o"]], d_attn.view(T, -1), ["o"], scale=sign, stream=main)
+        mark()
+        if s.inter:
+            sess.sgmv([d_y["up"]], d_y["o"], ["up"], scale=sign, stream=main)
+            mark()
+            sess.sgmv([d_y["down"]], d_y["up"], ["down"], scale=sign, stream=main)
+            mark()
+        if n_swap:
+            ev_side.record(side)
+            main.wait_event(ev_side)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    with torch.cuda.stream(main):
+        for k in range(args.warmup):
+            step(k)
+        barrier()
+        sampler = ClockSampler(local)
+        sampler.start()
+        evs = []
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(main)
+        for k in range(args.steps):
+            step(k, evs)
+        e1.record(main)
+        barrier()
+        clocks = sampler.result()
+        ms_total = e0.elapsed_time(e1)
+        # per-call device time from the events recorded between the calls of the timed steps
+        per = len(calls) + 1
+        call_ms = {c: 0.0 for c in calls}
+        for k in range(args.steps):
+            for j, c in enumerate(calls):
+                call_ms[c] += evs[k * per + j].elapsed_time(evs[k * per + j + 1])
+        call_ms = {c: v / args.steps for c, v in call_ms.items()}
+
+        # end to end: inputs start in pinned host memory, the result is read back, every step
+        def e2e_step(k):
+            d_x.view(torch.int16).copy_(h_x, non_blocking=True)
+            for m in names:
+                d_y[m].view(torch.int16).copy_(h_y[m], non_blocking=True)
+            step(0)
+            h_out.copy_(d_y["down" if s.inter else "o"].view(torch.int16), non_blocking=True)
+        e2e_steps = max(3, min(args.steps, 20))
+        for k in range(2):
+            e2e_step(k)
+        barrier()
+        f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        f0.record(main)
+        for k in range(e2e_steps):
+            e2e_step(k)
+        f1.record(main)
+        barrier()
+        ms_e2e = f0.elapsed_time(f1) / e2e_steps
+    flags = sess.status()["device_flags"]
+    t = torch.tensor([ms_total, ms_e2e], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_total, ms_e2e = float(t[0]), float(t[1])
+    ms_step = ms_total / args.steps
+    if rank == 0:
+        pk = peaks()
+        wm = work_model(wl)
+        kernels = {}
+        for c in calls:
+            w = wm[c]
+            sec = call_ms[c] * 1e-3
+            k = {"ms": round(call_ms[c], 4), "bound": w["bound"], "gbs": round(w["bytes"] / sec / 1e9, 1),
+                 "frac_hbm": round(w["bytes"] / sec / 1e9 / pk["hbm"], 4)}
+            if "flops" in w:
+                k["tflops"] = round(w["flops"] / sec / 1e12, 1)
+                k["frac_tensor"] = round(w["flops"] / sec / 1e12 / pk["tensor"], 4)
+            kernels[c] = k
+        top = max(calls, key=lambda c: call_ms[c])
+        w, sec = wm[top], call_ms[top] * 1e-3
+        if w["bound"] == "tensor":
+            ach, peak, unit = w["flops"] / sec / 1e12, pk["tensor"], "TFLOP/s"
+        else:
+            ach, peak, unit = w["bytes"] / sec / 1e9, pk["hbm"], "GB/s"
+        roof = {"kernel": top, "bound": w["bound"], "achieved": round(ach, 2), "peak": peak, "unit": unit,
+                "frac": round(ach / peak, 4), "traffic": None, "peak_source": pk["src"] + " (burst)",
+                "ms_per_launch": round(call_ms[top], 4)}
+        cb, _, _ = oracle_baseline(wl)
+        h2d = int(h_x.numel() * 2 + sum(h_y[m].numel() * 2 for m in names))
+        out = {
+            "metric": METRIC, "value": world * T / (ms_step * 1e-3), "unit": "tokens/s", "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": WORKLOAD_TEXT[args.workload], "new_tokens_per_step": T, "requests": wl.n_req,
+                       "distinct_adapters": len(wl.used_adapters()), "pool_blocks": wl.pool_blocks,
+                       "block_bytes": s.block_bytes, "swap_blocks_each_way": n_swap,
+                       "l2": "inputs larger than L2 (x, y and KV exceed 126 MB); no flush between steps",
+                       "parallelism": "independent batch per GPU, no collective"},
+            "roofline": roof, "kernels": kernels, "cpu_baseline": cb,
+            "e2e": {"value": world * T / (ms_e2e * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": h2d,
+                    "d2h_bytes_per_step": int(h_out.numel() * 2), "ms_per_step": ms_e2e},
+            "gpu_launches": launches_per_step * args.steps, "clocks": clocks, "device_flags": flags,
+        }
+        print(json.dumps(out))
+    sess.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def _rec(torch, stream):
+    e = torch.cuda.Event(enable_timing=True)
+    e.record(stream)
+    return e
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="prefill7b", choices=list(WORKLOAD_TEXT))
+    ap.add_argument("--swap-blocks", type=int, default=-1)
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    from paper_2505_03756_b200 import synth
+    wl = synth.make_workload(args.workload)
+    if args.impl == "reference":
+        run_reference(args, wl)
+    else:
+        run_ours(args, wl)
+
+
+if __name__ == "__main__":
+    main()

@@ -182,7 +182,10 @@ class Workload:
 
     # ---- tensors (float32 arrays holding bf16-representable values)
     def _normal(self, tag: str, shape, std: float) -> np.ndarray:
-        return round_bf16(Stream(self.seed, tag).normal(shape, std))
+        key = (tag, tuple(shape), std)
+        if key not in self._cache:
+            self._cache[key] = round_bf16(Stream(self.seed, tag).normal(shape, std))
+        return self._cache[key]
 
     def x(self, mat: str = "q") -> np.ndarray:
         """Layer input rows [T, d_in] for projection `mat` (q, k, v share one x)."""

@@ -96,6 +96,10 @@ int fl_pool_snapshot(fl_pool* pool, int host, uint32_t* free_ids, uint32_t cap, 
 /* Reads the sticky device flags (synchronises the device) and the counters.  clear != 0 resets the flags. */
 int fl_pool_status(fl_pool* pool, fl_status* out, int clear);
 int fl_last_cuda_error(fl_pool* pool);
+/* Tuning switches.  FL_OPT_PREFILL_KERNEL: 0 (default) = prefill attention on tcgen05 tensor cores with
+ * TMEM accumulators and TMA-staged pages; 1 = the mma.sync kernel (same results within rounding). */
+#define FL_OPT_PREFILL_KERNEL 1
+int fl_pool_set_option(fl_pool* pool, int key, int value);
 
 /* ---------------------------------------------------------------- adapters (Section 4.3)
  * "We perform block-wise partitioning of LoRAs along the rank dimension": an adapter is stored as
@@ -147,7 +151,9 @@ int fl_lora_sgmv_multi(fl_pool* pool, fl_bf16* const* ys, const fl_bf16* x, cons
  * prefix_lens[i] + j, i.e. block kv_tbl[kv_tbl_indptr[i] + pos / bt], slot pos % bt, where
  * bt = block_bytes / (2 * n_kv_heads * 128 * 2).  In-block layout: [K|V][kv_head][token][128] bf16.
  * req_indptr, kv_tbl_indptr [n_req+1], prefix_lens [n_req]: device int32; kv_tbl: device uint32.
- * The tables must already cover prefix_len + new tokens. */
+ * The tables must already cover prefix_len + new tokens.  The V slots behind a request's last token in
+ * its last block are set to zero (attention reads whole blocks; K/V stored by other means must keep
+ * unused slots finite). */
 int fl_kv_append(fl_pool* pool, const fl_bf16* k_new, const fl_bf16* v_new, const int32_t* req_indptr,
                  const int32_t* kv_tbl_indptr, const uint32_t* kv_tbl, const int32_t* prefix_lens,
                  int n_req, int n_tokens, int n_kv_heads, fl_stream stream);

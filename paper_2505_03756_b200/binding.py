@@ -54,6 +54,7 @@ _SIGS = {
     "fl_pool_snapshot": (C.c_int, [_vp, C.c_int, _vp, C.c_uint32, _u32p]),
     "fl_pool_status": (C.c_int, [_vp, C.POINTER(fl_status), C.c_int]),
     "fl_last_cuda_error": (C.c_int, [_vp]),
+    "fl_pool_set_option": (C.c_int, [_vp, C.c_int, C.c_int]),
     "fl_lora_blocks": (C.c_int, [C.c_size_t, C.c_int32, C.POINTER(fl_lora_shape), C.c_int, _u32p]),
     "fl_lora_pack_host": (C.c_int, [_vp, C.c_int32, C.POINTER(fl_lora_shape), C.c_int, C.POINTER(_vp),
                                     C.POINTER(_vp), _vp, C.c_uint32]),
@@ -182,6 +183,13 @@ def fl_pool_status(pool, clear=False):
 
 def fl_last_cuda_error(pool):
     return lib.fl_last_cuda_error(pool)
+
+
+FL_OPT_PREFILL_KERNEL = 1
+
+
+def fl_pool_set_option(pool, key, value):
+    _check(lib.fl_pool_set_option(pool, key, value), "fl_pool_set_option")
 
 
 def fl_lora_blocks(block_bytes, rank, mats):

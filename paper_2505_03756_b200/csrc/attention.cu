@@ -8,42 +8,14 @@
 // cores with an fp32 online softmax.
 #include <math.h>
 #include "mma_utils.cuh"
+#include "attention.cuh"
 #include "pool.cuh"
+
+using namespace attn;
 
 namespace {
 
-constexpr int D = FL_HEAD_DIM;
-constexpr int BT = 16;                 // tokens per block these kernels cover
-constexpr int PAGE_BYTES = BT * D * 2;   // one (block, kv head, K or V) piece
-constexpr int QT = 64;                 // query rows per prefill tile
-constexpr int KT = 64;                 // keys per prefill iteration
-constexpr int ATT_THREADS = 128;
-constexpr int DEC_ROWS = 16;
-
-struct PlanHdr {
-  int n_prefill, n_decode, chunk, pad;
-};
-
-struct AttnArgs {
-  PoolView pv;
-  __nv_bfloat16* out;
-  const __nv_bfloat16* q;
-  const int32_t* req_indptr;
-  const int32_t* tbl_indptr;
-  const uint32_t* tbl;
-  const int32_t* prefix_lens;
-  const int32_t* new_lens;
-  int n_req, n_q, n_kv;
-  float scale_log2;
-  // workspace
-  PlanHdr* hdr;
-  int2* prefill_list;   // (request, first query token of the tile inside the request)
-  int2* decode_list;    // (request, chunk)
-  int4* req_info;       // (first partial slot, chunks, decode?, 0)
-  float* part_o;        // [slot][kv head][16 rows][128]
-  float2* part_ml;      // [slot][kv head][16 rows] (running max in log2 units, sum)
-  int max_prefill, max_decode;
-};
+constexpr int QT = QT_MMA;
 
 __device__ __forceinline__ int block_excl_scan(int val, int* sh, int& total) {
   // exclusive scan over the 256 threads of the plan CTA
@@ -66,7 +38,7 @@ __device__ __forceinline__ int block_excl_scan(int val, int* sh, int& total) {
   return wbase + incl - val;
 }
 
-__global__ void __launch_bounds__(256) attn_plan_kernel(const AttnArgs a, int chunk) {
+__global__ void __launch_bounds__(256) attn_plan_kernel(const AttnArgs a, int chunk, int qt) {
   __shared__ int sh[8];
   const int group = a.n_q / a.n_kv;
   int base_p = 0, base_d = 0;
@@ -79,7 +51,7 @@ __global__ void __launch_bounds__(256) attn_plan_kernel(const AttnArgs a, int ch
       ctx = a.prefix_lens[i] + n;
       if (n > 0) {
         dec = n * group <= DEC_ROWS;
-        if (dec) chunks = (ctx + chunk - 1) / chunk; else tiles = (n + QT - 1) / QT;
+        if (dec) chunks = (ctx + chunk - 1) / chunk; else tiles = (n + qt - 1) / qt;
       }
     }
     int tot_p, tot_d;
@@ -88,7 +60,7 @@ __global__ void __launch_bounds__(256) attn_plan_kernel(const AttnArgs a, int ch
     if (i < a.n_req) {
       a.req_info[i] = make_int4(off_d, chunks, dec ? 1 : 0, 0);
       for (int t = 0; t < tiles; ++t)
-        if (off_p + t < a.max_prefill) a.prefill_list[off_p + t] = make_int2(i, t * QT);
+        if (off_p + t < a.max_prefill) a.prefill_list[off_p + t] = make_int2(i, t * qt);
       for (int c = 0; c < chunks; ++c)
         if (off_d + c < a.max_decode) a.decode_list[off_d + c] = make_int2(i, c);
     }
@@ -548,11 +520,14 @@ int fl_paged_attention(fl_pool* p, fl_bf16* out, const fl_bf16* q, const int32_t
       }
       configured[p->device & 15] = true;
     }
-    attn_plan_kernel<<<1, 256, 0, st>>>(a, w.chunk);
-    // a batch of n_tokens new tokens has at most max_prefill tiles; decode requests have one token
-    // row group each, so at most min(max_decode, ...) chunk items
-    if (w.max_prefill > 0 && n_tokens > 0)
+    const bool tc = p->prefill_kernel == 0;
+    attn_plan_kernel<<<1, 256, 0, st>>>(a, w.chunk, tc ? QT_TC : QT_MMA);
+    if (tc) {
+      rc = launch_prefill_tc(p, a, n_tokens, st);
+      if (rc != FL_OK) break;
+    } else {
       attn_prefill_kernel<<<(unsigned)w.max_prefill * n_q_heads, ATT_THREADS, PRE_SMEM, st>>>(a);
+    }
     attn_decode_kernel<<<(unsigned)w.max_decode * n_kv_heads, ATT_THREADS, DEC_SMEM, st>>>(a);
     attn_merge_kernel<<<(unsigned)n_req * n_kv_heads, ATT_THREADS, 0, st>>>(a);
     cudaError_t e = cudaGetLastError();

@@ -1,0 +1,45 @@
+// Declarations shared by the attention translation units.
+#pragma once
+#include "pool.cuh"
+
+namespace attn {
+
+constexpr int D = FL_HEAD_DIM;
+constexpr int BT = 16;                 // tokens per block these kernels cover
+constexpr int PAGE_BYTES = BT * D * 2;   // one (block, kv head, K or V) piece
+constexpr int QT_MMA = 64;             // query rows per prefill tile, mma.sync kernel
+constexpr int QT_TC = 128;             // query rows per prefill tile, tcgen05 kernel
+constexpr int KT = 64;                 // keys per prefill iteration
+constexpr int ATT_THREADS = 128;
+constexpr int DEC_ROWS = 16;
+
+struct PlanHdr {
+  int n_prefill, n_decode, chunk, pad;
+};
+
+struct AttnArgs {
+  PoolView pv;
+  __nv_bfloat16* out;
+  const __nv_bfloat16* q;
+  const int32_t* req_indptr;
+  const int32_t* tbl_indptr;
+  const uint32_t* tbl;
+  const int32_t* prefix_lens;
+  const int32_t* new_lens;
+  int n_req, n_q, n_kv;
+  float scale_log2;
+  // workspace
+  PlanHdr* hdr;
+  int2* prefill_list;   // (request, first query token of the tile inside the request)
+  int2* decode_list;    // (request, chunk)
+  int4* req_info;       // (first partial slot, chunks, decode?, 0)
+  float* part_o;        // [slot][kv head][16 rows][128]
+  float2* part_ml;      // [slot][kv head][16 rows] (running max in log2 units, sum)
+  int max_prefill, max_decode;
+};
+
+
+// Launches the tcgen05/TMEM prefill kernel over the plan's prefill list (tiles of QT_TC rows).
+int launch_prefill_tc(fl_pool* p, const AttnArgs& a, int n_tokens, cudaStream_t st);
+
+}  // namespace attn

@@ -222,6 +222,15 @@ int fl_pool_status(fl_pool* p, fl_status* out, int clear) {
 
 int fl_last_cuda_error(fl_pool* p) { return p ? p->last_cuda : 0; }
 
+int fl_pool_set_option(fl_pool* p, int key, int value) {
+  if (!p) return FL_EINVAL;
+  if (key == FL_OPT_PREFILL_KERNEL && (value == 0 || value == 1)) {
+    p->prefill_kernel = value;
+    return FL_OK;
+  }
+  return FL_EINVAL;
+}
+
 int fl_lora_blocks(size_t block_bytes, int32_t rank, const fl_lora_shape* mats, int n_mats, uint32_t* n_table) {
   if (!n_table || block_bytes == 0) return FL_EINVAL;
   return fl_layout_adapter(block_bytes, rank, mats, n_mats, nullptr, n_table);

@@ -71,6 +71,15 @@ __global__ void kv_append_kernel(PoolView pv, const uint4* __restrict__ k_new, c
     const uint4 val = (w ? v_new : k_new)[(size_t)t * per_side + r];
     dst[((size_t)(w * n_kv + h) * bt + slot) * CH + e] = val;
   }
+  // The request's last token also clears the V slots behind it in its block, so that attention can
+  // multiply those slots by a zero weight without meeting stale non-finite bit patterns.
+  if (t == req_indptr[i + 1] - 1 && slot + 1 < bt) {
+    const int rest = (bt - 1 - slot) * CH;
+    for (int c = threadIdx.x; c < n_kv * rest; c += blockDim.x) {
+      const int h = c / rest, r = c - h * rest;
+      dst[((size_t)(n_kv + h) * bt + slot + 1) * CH + r] = make_uint4(0u, 0u, 0u, 0u);
+    }
+  }
 }
 
 }  // namespace

@@ -233,9 +233,11 @@ def test_kv_append_bit_exact(H, name):
 
 
 # ------------------------------------------------------------------ a5/a6: attention
-def _attention_case(H, wl, sm_scale=None):
+def _attention_case(H, wl, sm_scale=None, prefill_kernel=0):
+    from paper_2505_03756_b200 import binding as fl
     s = H.Session(wl, adapters=[])
     try:
+        fl.fl_pool_set_option(s.pool, fl.FL_OPT_PREFILL_KERNEL, prefill_kernel)
         s.build_batch()
         s.fill_prefix_kv()
         k_new, v_new = wl.kv_new()
@@ -257,25 +259,34 @@ def _attention_case(H, wl, sm_scale=None):
         s.close()
 
 
+@pytest.mark.parametrize("kernel", [0, 1])
 @pytest.mark.parametrize("name", list(REDUCED))
-def test_attention_parity(H, name):
-    _attention_case(H, synth.make_workload(name, **REDUCED[name]))
+def test_attention_parity(H, name, kernel):
+    _attention_case(H, synth.make_workload(name, **REDUCED[name]), prefill_kernel=kernel)
 
 
-def test_attention_edges(H):
+def test_attention_sharp_softmax_rescales_accumulator(H):
+    # large logits that keep growing along the keys force the running maximum up tile after tile
+    wl = synth.make_workload("prefill7b", n_req=2, len_range=(300, 700))
+    _attention_case(H, wl, sm_scale=1.5)
+    _attention_case(H, wl, sm_scale=1.5, prefill_kernel=1)
+
+
+@pytest.mark.parametrize("kernel", [0, 1])
+def test_attention_edges(H, kernel):
     sh = synth.LayerShape(512, 4, 4)
     # no prefix, one token, ragged tails, a request with no new token, long decode context (several chunks)
     wl = synth.make_workload("tiny", n_req=6, len_range=(0, 0), n_adapters=1, shape=sh)
     wl.prefix_lens[:] = [0, 0, 17, 63, 1500, 40]
     wl.new_lens[:] = [1, 70, 1, 65, 1, 0]
     wl.pool_blocks = 256
-    _attention_case(H, wl)
+    _attention_case(H, wl, prefill_kernel=kernel)
     # grouped heads: decode rows = 2 tokens x 8 heads, and a sharp softmax
     sh = synth.LayerShape(1024, 16, 2)
     wl = synth.make_workload("tiny", n_req=3, len_range=(0, 0), n_adapters=1, shape=sh)
     wl.prefix_lens[:] = [300, 5, 0]
     wl.new_lens[:] = [2, 1, 130]
-    _attention_case(H, wl, sm_scale=0.5)
+    _attention_case(H, wl, sm_scale=0.5, prefill_kernel=kernel)
 
 
 def test_attention_prefix_reuse_equals_recompute_and_block_choice(H):

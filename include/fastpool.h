@@ -145,6 +145,29 @@ int fl_lora_sgmv_multi(fl_pool* pool, fl_bf16* const* ys, const fl_bf16* x, cons
                        const int32_t* seg_indptr, const int32_t* lora_ids, int n_seg, int n_tokens,
                        float scale, void* workspace, size_t workspace_bytes, fl_stream stream);
 
+/* fl_lora_sgmv without a workspace argument, for callers that cannot allocate device memory.  (The
+ * paper has no counterpart; this is a convenience of the library.)  A serving engine that follows the
+ * paper hands all of its HBM to the block pool at start-up; once it is serving, a cudaMalloc may fail
+ * for lack of memory, and even when it succeeds it stalls the whole device, so the step loop of such
+ * an engine (and any plug-in that is not allowed to touch the engine's memory budget) has nowhere to
+ * get the scratch that fl_lora_sgmv asks for.  This entry point brings its own: a fixed array of
+ * FL_SGMV_STATIC_BYTES that is part of the library image, so every GPU that loads the library holds
+ * that much memory until the process exits.  Neither this call nor anything it calls allocates or
+ * frees device or pinned memory.
+ *  - Same arguments, results and status codes as fl_lora_sgmv (one projection per call).
+ *  - Limit: FL_ENOMEM, with nothing launched, when fl_lora_sgmv_workspace(n_tokens, 1) exceeds
+ *    FL_SGMV_STATIC_BYTES; the 8 MiB cover every batch of up to 32767 tokens.
+ *  - The first call on a device looks up the array's device address (one runtime query, remembered
+ *    per device); make that first call outside any stream capture.
+ *  - All calls on one device share the array, and it keeps whatever the last call left in it.  The
+ *    kernels overwrite every value they later read, so nothing has to be cleared between calls, but two
+ *    calls whose kernels may overlap on the GPU (different streams without an ordering between them)
+ *    race on it: keep such calls on one stream or order them with events. */
+#define FL_SGMV_STATIC_BYTES (8u << 20)
+int fl_lora_sgmv_static(fl_pool* pool, fl_bf16* y, const fl_bf16* x, int mat_index,
+                        const int32_t* seg_indptr, const int32_t* lora_ids, int n_seg, int n_tokens,
+                        float scale, fl_stream stream);
+
 /* ---------------------------------------------------------------- KV store (Section 4.3: new KV stays in HBM blocks)
  * Writes the new tokens' K and V into the pool.  Request i owns tokens req_indptr[i] .. req_indptr[i+1]
  * of k_new / v_new (device, [n_tokens, n_kv_heads, 128] bf16); its token j goes to logical position

@@ -62,6 +62,7 @@ _SIGS = {
     "fl_lora_unregister": (C.c_int, [_vp, C.c_int32]),
     "fl_lora_sgmv_workspace": (C.c_size_t, [C.c_int, C.c_int]),
     "fl_lora_sgmv": (C.c_int, [_vp, _vp, _vp, C.c_int, _vp, _vp, C.c_int, C.c_int, C.c_float, _vp, C.c_size_t, _vp]),
+    "fl_lora_sgmv_static": (C.c_int, [_vp, _vp, _vp, C.c_int, _vp, _vp, C.c_int, C.c_int, C.c_float, _vp]),
     "fl_lora_sgmv_multi": (C.c_int, [_vp, C.POINTER(_vp), _vp, _i32p, C.c_int, _vp, _vp, C.c_int, C.c_int,
                                      C.c_float, _vp, C.c_size_t, _vp]),
     "fl_kv_append": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, C.c_int, C.c_int, C.c_int, _vp]),
@@ -225,6 +226,15 @@ def fl_lora_sgmv(pool, y, x, mat_index, seg_indptr, lora_ids, n_seg, n_tokens, s
     _check(lib.fl_lora_sgmv(pool, _dev(y), _dev(x), mat_index, _dev(seg_indptr), _dev(lora_ids), n_seg, n_tokens,
                             scale, _dev(workspace), workspace.numel() * workspace.element_size(), _stream(stream)),
            "fl_lora_sgmv")
+
+
+FL_SGMV_STATIC_BYTES = 8 << 20
+
+
+def fl_lora_sgmv_static(pool, y, x, mat_index, seg_indptr, lora_ids, n_seg, n_tokens, scale, stream=None):
+    """fl_lora_sgmv on the library's built-in scratch: the caller passes no workspace and nothing is allocated."""
+    _check(lib.fl_lora_sgmv_static(pool, _dev(y), _dev(x), mat_index, _dev(seg_indptr), _dev(lora_ids), n_seg,
+                                   n_tokens, scale, _stream(stream)), "fl_lora_sgmv_static")
 
 
 def fl_lora_sgmv_multi(pool, ys, x, mat_indices, seg_indptr, lora_ids, n_seg, n_tokens, scale, workspace, stream=None):

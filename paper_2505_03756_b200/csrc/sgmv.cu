@@ -437,4 +437,45 @@ int fl_lora_sgmv(fl_pool* p, fl_bf16* y, const fl_bf16* x, int mat_index,
                             workspace_bytes, stream);
 }
 
+// ---------------------------------------------------------------- fl_lora_sgmv_static: no allocation anywhere
+// The scratch that fl_lora_sgmv takes from its caller lives here instead, inside the library image.
+// Every GPU that loads the library holds these FL_SGMV_STATIC_BYTES until the process exits.
+}  // extern "C"
+
+static __device__ __align__(256) unsigned char g_sgmv_static_scratch[FL_SGMV_STATIC_BYTES];
+
+namespace {
+constexpr int STATIC_MAX_DEVICES = 64;
+void* g_static_scratch_addr[STATIC_MAX_DEVICES] = {};   // device address of the array, per device
+}  // namespace
+
+extern "C" {
+
+int fl_lora_sgmv_static(fl_pool* p, fl_bf16* y, const fl_bf16* x, int mat_index,
+                        const int32_t* seg_indptr, const int32_t* lora_ids, int n_seg, int n_tokens,
+                        float scale, fl_stream stream) {
+  if (!p || n_seg < 0 || n_tokens < 0) return FL_EINVAL;
+  if (p->device < 0 || p->device >= STATIC_MAX_DEVICES) return FL_EINVAL;
+  if (fl_lora_sgmv_workspace(n_tokens, 1) > (size_t)FL_SGMV_STATIC_BYTES) return FL_ENOMEM;   // batch too large for the built-in scratch
+  void* scratch = g_static_scratch_addr[p->device];
+  if (!scratch) {
+    // First call on this device: in host code the array's name is only a handle, so ask the runtime
+    // for the array's address on the pool's device (which must be current for the query).
+    int prev = -1;
+    cudaGetDevice(&prev);
+    if (prev != p->device) cudaSetDevice(p->device);
+    const cudaError_t e = cudaGetSymbolAddress(&scratch, g_sgmv_static_scratch);
+    if (prev != p->device && prev >= 0) cudaSetDevice(prev);
+    if (e != cudaSuccess || !scratch) {
+      p->last_cuda = (int)e;
+      return FL_ECUDA;
+    }
+    g_static_scratch_addr[p->device] = scratch;
+  }
+  // Nothing in the scratch has to start at zero: the shrink kernel writes every partial sum that the
+  // expand kernel reads, so whatever the previous call left behind is overwritten before use.
+  return fl_lora_sgmv(p, y, x, mat_index, seg_indptr, lora_ids, n_seg, n_tokens, scale, scratch,
+                      (size_t)FL_SGMV_STATIC_BYTES, stream);
+}
+
 }  // extern "C"

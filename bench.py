@@ -198,7 +198,7 @@ def run_ours(args, wl):
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     if rank > 0:      # requests are independent: every rank runs its own batch of the same shape (no exchange)
-        wl = synth.make_workload(args.workload, seed=wl.seed + 7919 * rank)
+        wl = synth.make_workload(args.workload, seed=wl.seed + 7919 * rank, **({"n_req": args.n_req} if args.n_req else {}))
     s = wl.shape
     T = wl.n_tokens
     n_swap = args.swap_blocks if args.swap_blocks >= 0 else (256 if args.workload == "swapstress" else 32)
@@ -368,10 +368,14 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="prefill7b", choices=list(WORKLOAD_TEXT))
     ap.add_argument("--swap-blocks", type=int, default=-1)
+    ap.add_argument("--n-req", type=int, default=0, help="reduced copy of the workload with this many requests "
+                    "(small pool; for profiler captures, not a bench line)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     from paper_2505_03756_b200 import synth
-    wl = synth.make_workload(args.workload)
+    wl = synth.make_workload(args.workload, n_req=args.n_req) if args.n_req else synth.make_workload(args.workload)
+    if args.n_req:
+        WORKLOAD_TEXT[args.workload] += f" -- REDUCED to {args.n_req} requests"
     if args.impl == "reference":
         run_reference(args, wl)
     else:

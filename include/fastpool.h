@@ -97,7 +97,9 @@ int fl_pool_snapshot(fl_pool* pool, int host, uint32_t* free_ids, uint32_t cap, 
 int fl_pool_status(fl_pool* pool, fl_status* out, int clear);
 int fl_last_cuda_error(fl_pool* pool);
 /* Tuning switches.  FL_OPT_PREFILL_KERNEL: 0 (default) = prefill attention on tcgen05 tensor cores with
- * TMEM accumulators and TMA-staged pages; 1 = the mma.sync kernel (same results within rounding). */
+ * TMEM accumulators and TMA-staged pages, two query tiles per CTA sharing the K/V stream; 1 = the
+ * mma.sync kernel; 2 = the tcgen05 kernel with one query tile per CTA.  Same results within rounding.
+ * The tcgen05 kernels need sm_scale > 0; other values are served by the mma.sync kernel. */
 #define FL_OPT_PREFILL_KERNEL 1
 int fl_pool_set_option(fl_pool* pool, int key, int value);
 

@@ -520,9 +520,13 @@ int fl_paged_attention(fl_pool* p, fl_bf16* out, const fl_bf16* q, const int32_t
       }
       configured[p->device & 15] = true;
     }
-    const bool tc = p->prefill_kernel == 0;
-    attn_plan_kernel<<<1, 256, 0, st>>>(a, w.chunk, tc ? QT_TC : QT_MMA);
-    if (tc) {
+    // the tensor-core kernels fold sm_scale into the exponent and take row maxima of raw scores: they need sm_scale > 0
+    const int kind = sm_scale > 0.f ? p->prefill_kernel : 1;
+    attn_plan_kernel<<<1, 256, 0, st>>>(a, w.chunk, kind == 0 ? tc2_tile_tokens(n_q_heads, n_kv_heads) : (kind == 2 ? QT_TC : QT_MMA));
+    if (kind == 0) {
+      rc = launch_prefill_tc2(p, a, n_tokens, w.max_prefill, st);
+      if (rc != FL_OK) break;
+    } else if (kind == 2) {
       rc = launch_prefill_tc(p, a, n_tokens, st);
       if (rc != FL_OK) break;
     } else {

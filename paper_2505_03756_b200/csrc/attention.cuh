@@ -2,6 +2,8 @@
 #pragma once
 #include "pool.cuh"
 
+struct CUtensorMap_st;
+
 namespace attn {
 
 constexpr int D = FL_HEAD_DIM;
@@ -39,7 +41,12 @@ struct AttnArgs {
 };
 
 
-// Launches the tcgen05/TMEM prefill kernel over the plan's prefill list (tiles of QT_TC rows).
+// Tensor maps of the pool slab (cached in the pool) and of q, as the tcgen05 prefill kernels read them.
+int prefill_tensor_maps(fl_pool* p, const AttnArgs& a, int n_tokens, const ::CUtensorMap_st** kv_out, ::CUtensorMap_st* qmap);
+// Launches the one-tile-per-CTA tcgen05/TMEM prefill kernel over the plan's prefill list (tiles of QT_TC rows).
 int launch_prefill_tc(fl_pool* p, const AttnArgs& a, int n_tokens, cudaStream_t st);
+// Launches the two-tiles-per-CTA kernel; the plan's tiles are tc2_tile_tokens(n_q, n_kv) tokens long.
+int launch_prefill_tc2(fl_pool* p, const AttnArgs& a, int n_tokens, int max_items, cudaStream_t st);
+inline int tc2_tile_tokens(int n_q, int n_kv) { return (n_q / n_kv) % 2 == 0 ? 128 : 256; }
 
 }  // namespace attn

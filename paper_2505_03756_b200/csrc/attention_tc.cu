@@ -18,9 +18,12 @@
 #include <string.h>
 #include "attention.cuh"
 #include "mma_utils.cuh"
+#include "tc_ptx.cuh"
 
 namespace attn {
 namespace {
+
+using namespace tc;
 
 constexpr int TC_THREADS = 192;
 constexpr int KT_TC = 64;
@@ -35,98 +38,9 @@ constexpr uint32_t OFF_BAR = OFF_P + QT_TC * KT_TC * 2;
 constexpr uint32_t TC_SMEM = OFF_BAR + 128;
 constexpr uint32_t TMEM_COLS = 256;               // S0 | S1 (64 each) | O (128)
 constexpr uint32_t TM_S = 0, TM_O = 128;
-constexpr uint32_t WAIT_LIMIT = 1u << 22;
 constexpr float RESCALE_STEP = 8.f;
 
 enum { B_QFULL = 0, B_KVFULL = 1, B_KVEMPTY = 3, B_SFULL = 5, B_SFREE = 7, B_PFULL = 9, B_PVDONE = 10, B_COUNT = 11 };
-
-// ---- PTX wrappers
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-  return ok != 0;
-}
-// Bounded wait: false when the CTA is aborting or the limit ran out (which raises the abort flag).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-  for (uint32_t i = 0; i < WAIT_LIMIT; ++i) {
-    if (mbar_try(bar, parity)) return true;
-    if ((i & 255u) == 255u && *abort_flag) return false;
-  }
-  *abort_flag = 1;
-  return false;
-}
-__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2, int c3) {
-  asm volatile(
-      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
-      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
-}
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2) {
-  asm volatile(
-      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
-      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
-}
-__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
-}
-__device__ __forceinline__ void umma_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-
-#define TM_REGS(r, o) \
-  "=r"(r[o + 0]), "=r"(r[o + 1]), "=r"(r[o + 2]), "=r"(r[o + 3]), "=r"(r[o + 4]), "=r"(r[o + 5]), "=r"(r[o + 6]), "=r"(r[o + 7])
-#define TM_IN(r, o) \
-  "r"(r[o + 0]), "r"(r[o + 1]), "r"(r[o + 2]), "r"(r[o + 3]), "r"(r[o + 4]), "r"(r[o + 5]), "r"(r[o + 6]), "r"(r[o + 7])
-
-// 32 consecutive TMEM columns of this thread's lane -> 32 registers (the warp reads its 32 lanes).
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-      : TM_REGS(r, 0), TM_REGS(r, 8), TM_REGS(r, 16), TM_REGS(r, 24)
-      : "r"(taddr) : "memory");
-}
-__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
-  asm volatile(
-      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
-      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
-      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
-      ::"r"(taddr), TM_IN(r, 0), TM_IN(r, 8), TM_IN(r, 16), TM_IN(r, 24) : "memory");
-}
-__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
-
-// Shared-memory matrix descriptor, 128-byte swizzle (layout code 2), descriptor version 1.
-// K-major operands: lbo unused (1), sbo = 1024 (8 rows of 128 bytes).  MN-major: lbo = distance
-// between 64-element groups along MN, sbo = 1024 (8 rows along K).
-__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
-  return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) | ((uint64_t)(sbo_bytes >> 4) << 32) |
-         (1ull << 46) | (2ull << 61);
-}
-// Instruction descriptor: fp32 accumulate, bf16 x bf16, M = 128, N = n; b_mn = B operand is MN-major.
-__host__ __device__ constexpr uint32_t instr_desc(int n, bool b_mn) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn ? 1u : 0u) << 16) | ((uint32_t)(n >> 3) << 17) | ((128u >> 4) << 24);
-}
 
 __global__ void __launch_bounds__(TC_THREADS, 2)
 attn_prefill_tc_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap kv_map, const __grid_constant__ CUtensorMap q_map) {
@@ -413,7 +327,7 @@ struct TmapCache {
 
 }  // namespace
 
-int launch_prefill_tc(fl_pool* p, const AttnArgs& a, int n_tokens, cudaStream_t st) {
+int prefill_tensor_maps(fl_pool* p, const AttnArgs& a, int n_tokens, const CUtensorMap** kv_out, CUtensorMap* qmap) {
   EncodeTiledFn enc = encode_fn();
   if (!enc) return FL_ECUDA;
   TmapCache* tc = reinterpret_cast<TmapCache*>(p->tmap_cache);
@@ -434,17 +348,24 @@ int launch_prefill_tc(fl_pool* p, const AttnArgs& a, int n_tokens, cudaStream_t 
     }
     tc->n_kv = a.n_kv;
   }
+  // q as [token][head][128]: box = 64 elements x 128 tokens of one head
+  const cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)a.n_q, (cuuint64_t)n_tokens};
+  const cuuint64_t strides[2] = {(cuuint64_t)D * 2, (cuuint64_t)a.n_q * D * 2};
+  const cuuint32_t box[3] = {64, 1, (cuuint32_t)QT_TC};
+  const cuuint32_t es[3] = {1, 1, 1};
+  if (enc(qmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<__nv_bfloat16*>(a.q), dims, strides, box, es,
+          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+    return FL_ECUDA;
+  *kv_out = &tc->kv;
+  return FL_OK;
+}
+
+int launch_prefill_tc(fl_pool* p, const AttnArgs& a, int n_tokens, cudaStream_t st) {
+  const CUtensorMap* kv = nullptr;
   alignas(64) CUtensorMap qmap;
-  {
-    const cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)a.n_q, (cuuint64_t)n_tokens};
-    const cuuint64_t strides[2] = {(cuuint64_t)D * 2, (cuuint64_t)a.n_q * D * 2};
-    const cuuint32_t box[3] = {64, 1, (cuuint32_t)QT_TC};
-    const cuuint32_t es[3] = {1, 1, 1};
-    if (enc(&qmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<__nv_bfloat16*>(a.q), dims, strides, box, es,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-      return FL_ECUDA;
-  }
+  int rc = prefill_tensor_maps(p, a, n_tokens, &kv, &qmap);
+  if (rc != FL_OK) return rc;
   static bool configured[16] = {};
   if (!configured[p->device & 15]) {
     FL_CUDA(p, cudaFuncSetAttribute(attn_prefill_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TC_SMEM));
@@ -452,7 +373,7 @@ int launch_prefill_tc(fl_pool* p, const AttnArgs& a, int n_tokens, cudaStream_t 
   }
   // tiles of 128 rows: at most n_tokens / 128 + n_req of them
   const unsigned tiles = (unsigned)(n_tokens / QT_TC + a.n_req);
-  attn_prefill_tc_kernel<<<tiles * a.n_q, TC_THREADS, TC_SMEM, st>>>(a, tc->kv, qmap);
+  attn_prefill_tc_kernel<<<tiles * a.n_q, TC_THREADS, TC_SMEM, st>>>(a, *kv, qmap);
   FL_CUDA(p, cudaGetLastError());
   return FL_OK;
 }

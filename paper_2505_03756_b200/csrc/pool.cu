@@ -224,7 +224,7 @@ int fl_last_cuda_error(fl_pool* p) { return p ? p->last_cuda : 0; }
 
 int fl_pool_set_option(fl_pool* p, int key, int value) {
   if (!p) return FL_EINVAL;
-  if (key == FL_OPT_PREFILL_KERNEL && (value == 0 || value == 1)) {
+  if (key == FL_OPT_PREFILL_KERNEL && value >= 0 && value <= 2) {
     p->prefill_kernel = value;
     return FL_OK;
   }

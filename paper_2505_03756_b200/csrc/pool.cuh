@@ -67,7 +67,7 @@ struct fl_pool {
   uint64_t bytes_in = 0, bytes_out = 0;
   int last_cuda = 0;
   int sm_count = 148;
-  int prefill_kernel = 0;                           // 0: tcgen05/TMEM kernel, 1: mma.sync kernel
+  int prefill_kernel = 0;                           // 0: tcgen05 two-tile kernel, 1: mma.sync kernel, 2: tcgen05 one-tile kernel
   void* tmap_cache = nullptr;                      // tensor maps of the slab, keyed by KV head count
   PoolView view() const { return PoolView{slab, block_bytes, n_blocks, d_dir, dir_cap, d_tables, d_flags}; }
 };

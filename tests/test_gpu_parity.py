@@ -259,7 +259,7 @@ def _attention_case(H, wl, sm_scale=None, prefill_kernel=0):
         s.close()
 
 
-@pytest.mark.parametrize("kernel", [0, 1])
+@pytest.mark.parametrize("kernel", [0, 1, 2])
 @pytest.mark.parametrize("name", list(REDUCED))
 def test_attention_parity(H, name, kernel):
     _attention_case(H, synth.make_workload(name, **REDUCED[name]), prefill_kernel=kernel)
@@ -268,11 +268,11 @@ def test_attention_parity(H, name, kernel):
 def test_attention_sharp_softmax_rescales_accumulator(H):
     # large logits that keep growing along the keys force the running maximum up tile after tile
     wl = synth.make_workload("prefill7b", n_req=2, len_range=(300, 700))
-    _attention_case(H, wl, sm_scale=1.5)
-    _attention_case(H, wl, sm_scale=1.5, prefill_kernel=1)
+    for kernel in (0, 1, 2):
+        _attention_case(H, wl, sm_scale=1.5, prefill_kernel=kernel)
 
 
-@pytest.mark.parametrize("kernel", [0, 1])
+@pytest.mark.parametrize("kernel", [0, 1, 2])
 def test_attention_edges(H, kernel):
     sh = synth.LayerShape(512, 4, 4)
     # no prefix, one token, ragged tails, a request with no new token, long decode context (several chunks)

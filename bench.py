@@ -226,10 +226,11 @@ def run_ours(args, wl):
     spare = int(np.sum((wl.new_lens + s.block_tokens - 1) // s.block_tokens))
     spare = min(spare, fl.fl_pool_status(sess.pool)["blocks_free"])
     main = torch.cuda.Stream()
-    side = torch.cuda.Stream()
-    ev_side = torch.cuda.Event()
+    side, side_in = torch.cuda.Stream(), torch.cuda.Stream()      # swap-out and swap-in overlap each other too
+    ev_side, ev_side_in = torch.cuda.Event(), torch.cuda.Event()
     calls = ["sgmv_qkv", "kv_append", "attention", "sgmv_o"] + (["sgmv_up", "sgmv_down"] if s.inter else [])
-    launches_per_step = 2 + 1 + 4 + 2 + (4 if s.inter else 0)
+    # shrink + expand per SGMV call, KV append, plan + prefill + decode + merge, swap gather + scatter
+    launches_per_step = 2 + 1 + 4 + 2 + (4 if s.inter else 0) + (2 * -(-n_swap // 256) if n_swap > 1 else 0)
 
     def step(k, evs=None):
         sign = wl.scale if k % 2 == 0 else -wl.scale     # y += s*delta, then y -= s*delta: values stay bounded
@@ -237,7 +238,7 @@ def run_ours(args, wl):
         fl.fl_block_free(sess.pool, ids[::-1])
         if n_swap:                                        # a7: side stream, overlapped
             fl.fl_swap_out(sess.pool, swap_dev_out, swap_host_out, side)
-            fl.fl_swap_in(sess.pool, swap_dev_in, swap_host_in, side)
+            fl.fl_swap_in(sess.pool, swap_dev_in, swap_host_in, side_in)
         mark = (lambda: None) if evs is None else (lambda: evs.append(_rec(torch, main)))
         mark()
         sess.sgmv([d_y["q"], d_y["k"], d_y["v"]], d_x, ["q", "k", "v"], scale=sign, stream=main)
@@ -255,7 +256,9 @@ def run_ours(args, wl):
             mark()
         if n_swap:
             ev_side.record(side)
+            ev_side_in.record(side_in)
             main.wait_event(ev_side)
+            main.wait_event(ev_side_in)
 
     def barrier():
         torch.cuda.synchronize()
@@ -304,6 +307,45 @@ def run_ours(args, wl):
         f1.record(main)
         barrier()
         ms_e2e = f0.elapsed_time(f1) / e2e_steps
+        # the swap alone (both directions at once), and the host link's own peak for the same byte count
+        swap = None
+        if n_swap:
+            def swap_once():
+                fl.fl_swap_out(sess.pool, swap_dev_out, swap_host_out, side)
+                fl.fl_swap_in(sess.pool, swap_dev_in, swap_host_in, side_in)
+                ev_side.record(side)
+                ev_side_in.record(side_in)
+                main.wait_event(ev_side)
+                main.wait_event(ev_side_in)
+            nbytes = n_swap * s.block_bytes
+            hp = torch.empty(2 * nbytes, dtype=torch.uint8).pin_memory()
+            dp = torch.empty(2 * nbytes, dtype=torch.uint8, device=dev)
+
+            def link_once():
+                with torch.cuda.stream(side):
+                    hp[:nbytes].copy_(dp[:nbytes], non_blocking=True)
+                with torch.cuda.stream(side_in):
+                    dp[nbytes:].copy_(hp[nbytes:], non_blocking=True)
+                ev_side.record(side)
+                ev_side_in.record(side_in)
+                main.wait_event(ev_side)
+                main.wait_event(ev_side_in)
+            res = {}
+            for name, fn in (("swap", swap_once), ("link", link_once)):
+                fn()
+                barrier()
+                g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                g0.record(main)
+                for _ in range(5):
+                    fn()
+                g1.record(main)
+                barrier()
+                res[name] = g0.elapsed_time(g1) / 5
+            swap = {"ms": round(res["swap"], 4), "bytes_each_way": nbytes, "bound": "host link",
+                    "gbs_each_way": round(nbytes / res["swap"] / 1e6, 2),
+                    "link_peak_gbs_each_way": round(nbytes / res["link"] / 1e6, 2),
+                    "frac_link": round(res["link"] / res["swap"], 4),
+                    "note": "both directions at once; peak = two contiguous pinned copies of the same size, measured here"}
     flags = sess.status()["device_flags"]
     t = torch.tensor([ms_total, ms_e2e], dtype=torch.float64, device=dev)
     if world > 1:
@@ -323,6 +365,8 @@ def run_ours(args, wl):
                 k["tflops"] = round(w["flops"] / sec / 1e12, 1)
                 k["frac_tensor"] = round(w["flops"] / sec / 1e12 / pk["tensor"], 4)
             kernels[c] = k
+        if swap:
+            kernels["swap"] = swap
         top = max(calls, key=lambda c: call_ms[c])
         w, sec = wm[top], call_ms[top] * 1e-3
         if w["bound"] == "tensor":

@@ -201,9 +201,15 @@ int fl_paged_attention(fl_pool* pool, fl_bf16* out, const fl_bf16* q, const int3
 
 /* ---------------------------------------------------------------- swap (Section 4.3 "Asynchronous Swapping-in/out")
  * Copies whole blocks between the device slab and the pinned host slab, pair k = (dev_ids[k],
- * host_ids[k]) (host pointers), in list order, asynchronously on `side` (copy engines), so that it
- * overlaps kernels running on other streams.  Every listed block must be allocated (FL_EBADID,
- * nothing copied).  The caller guarantees that no kernel in flight touches the listed device blocks
+ * host_ids[k]) (host pointers), asynchronously on `side`, so that it overlaps kernels running on other
+ * streams.  Every listed block must be allocated (FL_EBADID) and no block may be listed twice in one
+ * call (FL_EINVAL); on either error nothing is copied.  The transfers run on the copy engines: pairs
+ * that are consecutive in both memories go as one DMA; a run of consecutive host blocks whose device
+ * blocks are scattered goes through a staging area inside the pool (one small gather or scatter kernel
+ * on `side` plus one DMA for up to 256 blocks), which is what a fragmented pool needs to keep the host
+ * link busy.  Swap-out and swap-in have separate staging areas, so the two directions overlap when they
+ * are given different streams; calls in one direction are ordered among themselves by the library even
+ * across streams.  The caller guarantees that no kernel in flight touches the listed device blocks
  * (the paper evicts only nodes no running query uses, and a query whose blocks are in flight waits).
  * fl_swap_record records `ev` on the side stream; fl_swap_wait polls it on the host until done or
  * timeout_ms elapsed (FL_ETIMEOUT) - no device-side waiting. */

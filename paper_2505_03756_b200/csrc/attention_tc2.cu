@@ -40,6 +40,10 @@ constexpr uint32_t OFF_BAR2 = OFF_RING + NSLOT * TILE_BYTES;
 constexpr uint32_t T2_SMEM = OFF_BAR2 + 256;
 constexpr uint32_t T2_TMEM_COLS = 512;                 // S_A | S_B | O_A | O_B, 128 columns each
 constexpr float RESCALE_LOG2 = 8.f;
+#ifndef FL_POLY_OF_4
+#define FL_POLY_OF_4 0
+#endif
+constexpr int POLY_OF_4 = FL_POLY_OF_4;
 
 enum { C_QFULL = 0, C_FULL = 1, C_EMPTY = C_FULL + NSLOT, C_SFULL = C_EMPTY + NSLOT, C_PFULL = C_SFULL + 2,
        C_ODONE = C_PFULL + 2, C_COUNT = C_ODONE + 2 };
@@ -281,7 +285,9 @@ attn_prefill_tc2_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap kv
 #pragma unroll
         for (int e = 0; e < 16; ++e) {
           const float2 arg = __ffma2_rn(make_float2(__uint_as_float(s[c][2 * e]), __uint_as_float(s[c][2 * e + 1])), sc2, nm2);
-          const float2 p = make_float2(ex2_approx(arg.x), ex2_approx(arg.y));
+          // POLY_OF_4 of every 4 pairs take the polynomial, the others the special-function unit: the two
+          // run side by side and the slower unit no longer sets the pace of the tile
+          const float2 p = (e & 3) < POLY_OF_4 ? ex2_poly2(arg) : make_float2(ex2_approx(arg.x), ex2_approx(arg.y));
           sum[e & 1] = __fadd2_rn(sum[e & 1], p);
           pk[e] = pack_bf16(p.x, p.y);
         }

@@ -128,6 +128,14 @@ int fl_pool_create(fl_pool** out, size_t block_bytes, uint32_t n_blocks, uint32_
   if (e == cudaSuccess) e = cudaMalloc(&p->d_tables, sizeof(uint32_t) * (size_t)p->tables_cap);
   if (e == cudaSuccess) e = cudaMalloc(&p->d_flags, 64);
   if (e == cudaSuccess) e = cudaMemset(p->d_flags, 0, 64);
+  if (e == cudaSuccess && n_host_blocks > 1) {
+    // staging areas of the swap path: up to 256 blocks per direction
+    p->stage_blocks = std::min(256u, std::min(n_blocks, n_host_blocks));
+    for (int d = 0; d < 2 && e == cudaSuccess; ++d) {
+      e = cudaMalloc(&p->stage[d], (size_t)p->stage_blocks * block_bytes);
+      if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->stage_done[d], cudaEventDisableTiming);
+    }
+  }
   if (e == cudaSuccess) e = cudaDeviceGetAttribute(&p->sm_count, cudaDevAttrMultiProcessorCount, device);
   if (e != cudaSuccess) {
     cudaGetLastError();
@@ -150,6 +158,10 @@ int fl_pool_destroy(fl_pool* p) {
   if (p->d_dir) cudaFree(p->d_dir);
   if (p->d_tables) cudaFree(p->d_tables);
   if (p->d_flags) cudaFree(p->d_flags);
+  for (int d = 0; d < 2; ++d) {
+    if (p->stage[d]) cudaFree(p->stage[d]);
+    if (p->stage_done[d]) cudaEventDestroy(p->stage_done[d]);
+  }
   if (p->tmap_cache) free(p->tmap_cache);
   delete p;
   return FL_OK;

@@ -68,6 +68,9 @@ struct fl_pool {
   int last_cuda = 0;
   int sm_count = 148;
   int prefill_kernel = 0;                           // 0: tcgen05 two-tile kernel, 1: mma.sync kernel, 2: tcgen05 one-tile kernel
+  unsigned char* stage[2] = {nullptr, nullptr};     // contiguous staging areas of the swap path (out, in)
+  uint32_t stage_blocks = 0;
+  cudaEvent_t stage_done[2] = {nullptr, nullptr};   // last use of each staging area
   void* tmap_cache = nullptr;                      // tensor maps of the slab, keyed by KV head count
   PoolView view() const { return PoolView{slab, block_bytes, n_blocks, d_dir, dir_cap, d_tables, d_flags}; }
 };

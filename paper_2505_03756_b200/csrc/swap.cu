@@ -1,36 +1,119 @@
 // Block swap between the pinned host slab and the device slab, on a side stream (copy engines),
 // and the KV store kernel that writes new tokens' K,V into pool blocks.
+#include <algorithm>
 #include <chrono>
 #include <thread>
+#include <vector>
 #include "pool.cuh"
 
 namespace {
 
+constexpr uint32_t STAGE_CHUNK = 512;            // block ids per gather/scatter launch (passed by value)
+struct IdChunk { uint32_t ids[STAGE_CHUNK]; };
+
+// Copies whole pool blocks between the slab and a contiguous staging area: block ch.ids[k] <-> stage
+// block k.  blockIdx.x = k * parts + part; every CTA moves one slice of one block with 16-byte accesses.
+__global__ void __launch_bounds__(256) block_stage_kernel(unsigned char* __restrict__ slab, unsigned char* __restrict__ stage,
+                                                          const __grid_constant__ IdChunk ch, uint32_t u4_per_block,
+                                                          uint32_t parts, uint32_t n_pool_blocks, int to_stage,
+                                                          uint32_t* __restrict__ flags) {
+  const uint32_t k = blockIdx.x / parts, part = blockIdx.x % parts;
+  const uint32_t blk = ch.ids[k];
+  if (blk >= n_pool_blocks) {
+    if (threadIdx.x == 0) atomicOr(flags, (uint32_t)FLAG_BAD_BLOCK);
+    return;
+  }
+  const uint32_t per = (u4_per_block + parts - 1) / parts;
+  const uint32_t lo = part * per, hi = min(u4_per_block, lo + per);
+  uint4* pool_blk = reinterpret_cast<uint4*>(slab) + (size_t)blk * u4_per_block;
+  uint4* stage_blk = reinterpret_cast<uint4*>(stage) + (size_t)k * u4_per_block;
+  const uint4* src = to_stage ? pool_blk : stage_blk;
+  uint4* dst = to_stage ? stage_blk : pool_blk;
+  uint32_t i = lo + threadIdx.x;
+  for (; i + 3 * 256 < hi; i += 4 * 256) {       // four independent 16-byte loads in flight per thread
+    const uint4 a = src[i], b = src[i + 256], c = src[i + 512], d = src[i + 768];
+    dst[i] = a; dst[i + 256] = b; dst[i + 512] = c; dst[i + 768] = d;
+  }
+  for (; i < hi; i += 256) dst[i] = src[i];
+}
+
+// Swap of the listed (device block, host block) pairs on stream `side`.  Runs of consecutive host blocks
+// whose device blocks are scattered over the pool go through a contiguous staging area in device memory:
+// one gather kernel + one DMA per run (swap-out), or one DMA + one scatter kernel (swap-in), so the copy
+// engine moves a few large pieces instead of one small piece per block.  Everything else is one DMA per
+// run of pairs consecutive in both memories.
 int swap_blocks(fl_pool* p, const uint32_t* dev_ids, const uint32_t* host_ids, uint32_t n, fl_stream side, bool in) {
   if (!p || (n && (!dev_ids || !host_ids))) return FL_EINVAL;
-  for (uint32_t k = 0; k < n; ++k) {
-    if (dev_ids[k] >= p->n_blocks || !p->dev.used[dev_ids[k]]) return FL_EBADID;
-    if (host_ids[k] >= p->n_host_blocks || !p->host.used[host_ids[k]]) return FL_EBADID;
+  // validate everything before the first copy: range, allocated, no block listed twice
+  int bad = FL_OK;
+  uint32_t marked = 0;
+  for (; marked < n; ++marked) {
+    const uint32_t d = dev_ids[marked], h = host_ids[marked];
+    if (d >= p->n_blocks || h >= p->n_host_blocks || !p->dev.used[d] || !p->host.used[h]) { bad = FL_EBADID; break; }
+    if (p->dev.used[d] == 2 || p->host.used[h] == 2) { bad = FL_EINVAL; break; }
+    p->dev.used[d] = 2;
+    p->host.used[h] = 2;
   }
+  for (uint32_t k = 0; k < marked; ++k) p->dev.used[dev_ids[k]] = p->host.used[host_ids[k]] = 1;
+  if (bad != FL_OK) return bad;
+  if (n == 0) return FL_OK;
   int prev = -1;
   cudaGetDevice(&prev);
   if (prev != p->device) cudaSetDevice(p->device);
-  int rc = FL_OK;
-  // one DMA per run of pairs that are consecutive in both memories
-  for (uint32_t k = 0; k < n;) {
-    uint32_t run = 1;
-    while (k + run < n && dev_ids[k + run] == dev_ids[k] + run && host_ids[k + run] == host_ids[k] + run) ++run;
-    unsigned char* d = p->slab + (size_t)dev_ids[k] * p->block_bytes;
-    unsigned char* h = p->host_slab + (size_t)host_ids[k] * p->block_bytes;
-    cudaError_t e = in ? cudaMemcpyAsync(d, h, run * p->block_bytes, cudaMemcpyHostToDevice, (cudaStream_t)side)
-                       : cudaMemcpyAsync(h, d, run * p->block_bytes, cudaMemcpyDeviceToHost, (cudaStream_t)side);
-    if (e != cudaSuccess) {
-      p->last_cuda = (int)e;
-      rc = FL_ECUDA;
-      break;
+  const cudaStream_t st = (cudaStream_t)side;
+  const size_t bb = p->block_bytes;
+  std::vector<uint32_t> order(n);
+  for (uint32_t k = 0; k < n; ++k) order[k] = k;
+  std::sort(order.begin(), order.end(), [&](uint32_t a, uint32_t b) { return host_ids[a] < host_ids[b]; });
+  const int dir = in ? 1 : 0;
+  const uint32_t u4 = (uint32_t)(bb / 16);
+  const uint32_t parts = std::max(1u, std::min(32u, u4 / 1024));
+  bool staged_any = false;
+  cudaError_t e = cudaSuccess;
+  for (uint32_t k = 0; k < n && e == cudaSuccess;) {
+    uint32_t run = 1, both = 1;
+    while (k + run < n && host_ids[order[k + run]] == host_ids[order[k]] + run) {
+      if (both == run && dev_ids[order[k + run]] == dev_ids[order[k]] + run) ++both;
+      ++run;
     }
-    (in ? p->bytes_in : p->bytes_out) += (uint64_t)run * p->block_bytes;
-    k += run;
+    unsigned char* h = p->host_slab + (size_t)host_ids[order[k]] * bb;
+    if (both > 1 || run == 1 || !p->stage[dir]) {
+      // pairs consecutive in both memories (or a lone block): one DMA
+      const uint32_t len = both;
+      unsigned char* d = p->slab + (size_t)dev_ids[order[k]] * bb;
+      e = in ? cudaMemcpyAsync(d, h, len * bb, cudaMemcpyHostToDevice, st) : cudaMemcpyAsync(h, d, len * bb, cudaMemcpyDeviceToHost, st);
+      k += len;
+      continue;
+    }
+    // scattered device blocks, consecutive host blocks: through the staging area, STAGE_CHUNK blocks at most per piece
+    const uint32_t len = std::min(run, std::min(p->stage_blocks, STAGE_CHUNK));
+    if (!staged_any) {
+      e = cudaStreamWaitEvent(st, p->stage_done[dir], 0);   // the staging area may still be in use on another stream
+      if (e != cudaSuccess) break;
+      staged_any = true;
+    }
+    IdChunk ch;
+    for (uint32_t i = 0; i < len; ++i) ch.ids[i] = dev_ids[order[k + i]];
+    if (in) {
+      e = cudaMemcpyAsync(p->stage[dir], h, len * bb, cudaMemcpyHostToDevice, st);
+      if (e == cudaSuccess) {
+        block_stage_kernel<<<len * parts, 256, 0, st>>>(p->slab, p->stage[dir], ch, u4, parts, p->n_blocks, 0, p->d_flags);
+        e = cudaGetLastError();
+      }
+    } else {
+      block_stage_kernel<<<len * parts, 256, 0, st>>>(p->slab, p->stage[dir], ch, u4, parts, p->n_blocks, 1, p->d_flags);
+      e = cudaGetLastError();
+      if (e == cudaSuccess) e = cudaMemcpyAsync(h, p->stage[dir], len * bb, cudaMemcpyDeviceToHost, st);
+    }
+    k += len;
+  }
+  if (staged_any && e == cudaSuccess) e = cudaEventRecord(p->stage_done[dir], st);
+  int rc = FL_OK;
+  if (e != cudaSuccess) {
+    p->last_cuda = (int)e;
+    rc = FL_ECUDA;
+  } else {
+    (in ? p->bytes_in : p->bytes_out) += (uint64_t)n * bb;
   }
   if (prev != p->device && prev >= 0) cudaSetDevice(prev);
   return rc;

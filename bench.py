@@ -185,6 +185,27 @@ def run_reference(args, wl):
         "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
 
 
+def rank_workload(name, base_seed, rank, n_req=0):
+    """Requests are independent, so rank r runs its own batch of the same shape, drawn from its own seed."""
+    from paper_2505_03756_b200 import synth
+    kw = {"n_req": n_req} if n_req else {}
+    if rank == 0:
+        return synth.make_workload(name, **kw)
+    return synth.make_workload(name, seed=base_seed + 7919 * rank, **kw)
+
+
+def reduce_over_ranks(times_ms, tokens, world, device):
+    """Job-level numbers from per-rank ones: every time is the maximum over ranks, tokens are summed."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(list(times_ms), dtype=torch.float64, device=device)
+    n = torch.tensor([tokens], dtype=torch.int64, device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        dist.all_reduce(n, op=dist.ReduceOp.SUM)
+    return [float(v) for v in t], int(n[0])
+
+
 # ------------------------------------------------------------------ the CUDA leg
 def run_ours(args, wl):
     import torch
@@ -197,12 +218,11 @@ def run_ours(args, wl):
     torch.cuda.set_device(local)
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-    if rank > 0:      # requests are independent: every rank runs its own batch of the same shape (no exchange)
-        wl = synth.make_workload(args.workload, seed=wl.seed + 7919 * rank, **({"n_req": args.n_req} if args.n_req else {}))
+    wl = rank_workload(args.workload, wl.seed, rank, args.n_req)   # no exchange between ranks
     s = wl.shape
     T = wl.n_tokens
     n_swap = args.swap_blocks if args.swap_blocks >= 0 else (256 if args.workload == "swapstress" else 32)
-    sess = H.Session(wl, device=local, extra_host_blocks=2 * n_swap)
+    sess = H.Session(wl, device=local, extra_host_blocks=2 * n_swap, register_all=(args.workload == "swapstress"))
     sess.load_adapters()
     # the new-token blocks are taken and returned every step (allocator on the path); tables stay put
     sess.build_batch()
@@ -347,10 +367,7 @@ def run_ours(args, wl):
                     "frac_link": round(res["link"] / res["swap"], 4),
                     "note": "both directions at once; peak = two contiguous pinned copies of the same size, measured here"}
     flags = sess.status()["device_flags"]
-    t = torch.tensor([ms_total, ms_e2e], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_total, ms_e2e = float(t[0]), float(t[1])
+    (ms_total, ms_e2e), tokens_all = reduce_over_ranks([ms_total, ms_e2e], T, world, dev)
     ms_step = ms_total / args.steps
     if rank == 0:
         pk = peaks()
@@ -379,7 +396,7 @@ def run_ours(args, wl):
         cb, _, _ = oracle_baseline(wl)
         h2d = int(h_x.numel() * 2 + sum(h_y[m].numel() * 2 for m in names))
         out = {
-            "metric": METRIC, "value": world * T / (ms_step * 1e-3), "unit": "tokens/s", "n_gpus": world,
+            "metric": METRIC, "value": tokens_all / (ms_step * 1e-3), "unit": "tokens/s", "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": WORKLOAD_TEXT[args.workload], "new_tokens_per_step": T, "requests": wl.n_req,
@@ -388,7 +405,7 @@ def run_ours(args, wl):
                        "l2": "inputs larger than L2 (x, y and KV exceed 126 MB); no flush between steps",
                        "parallelism": "independent batch per GPU, no collective"},
             "roofline": roof, "kernels": kernels, "cpu_baseline": cb,
-            "e2e": {"value": world * T / (ms_e2e * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": h2d,
+            "e2e": {"value": tokens_all / (ms_e2e * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": int(h_out.numel() * 2), "ms_per_step": ms_e2e},
             "gpu_launches": launches_per_step * args.steps, "clocks": clocks, "device_flags": flags,
         }

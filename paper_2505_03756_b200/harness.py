@@ -33,7 +33,10 @@ def dev_to_f32(t: torch.Tensor) -> np.ndarray:
 
 class Session:
     def __init__(self, wl: synth.Workload, device: int = 0, scramble: bool = True, extra_host_blocks: int = 0,
-                 adapters=None):
+                 adapters=None, register_all: bool = False):
+        """adapters: ids to load (default: the ones the batch uses).  register_all: every adapter of the
+        workload is packed, swapped in and registered; those the batch never touches get filler weights
+        (one shared noise pattern), since drawing a thousand adapters value by value takes minutes."""
         self.wl = wl
         self.shape = wl.shape
         self.dev = torch.device("cuda", device)
@@ -43,6 +46,10 @@ class Session:
         self.block_bytes = wl.shape.block_bytes
         self.bt = wl.shape.block_tokens
         self.adapter_ids = wl.used_adapters() if adapters is None else list(adapters)
+        self.filler_ids = set()
+        if register_all:
+            self.filler_ids = set(range(len(wl.ranks))) - set(self.adapter_ids)
+            self.adapter_ids = list(range(len(wl.ranks)))
         self.n_table = {a: fl.fl_lora_blocks(self.block_bytes, int(wl.ranks[a]), self.mats) for a in self.adapter_ids}
         self.n_host_blocks = sum(self.n_table.values()) + extra_host_blocks
         self.pool = fl.fl_pool_create(self.block_bytes, wl.pool_blocks, max(1, self.n_host_blocks), device)
@@ -79,7 +86,11 @@ class Session:
         for a in self.adapter_ids:
             rank = int(self.wl.ranks[a])
             A, B = [], []
-            for name, _, _ in self.shape.mats:
+            for name, d_in, d_out in self.shape.mats:
+                if a in self.filler_ids:
+                    A.append(self._filler(d_in * rank).reshape(d_in, rank))
+                    B.append(self._filler(rank * d_out).reshape(rank, d_out))
+                    continue
                 am, bm = self.wl.adapter(a, name)
                 A.append(synth.bf16_bits(am))
                 B.append(synth.bf16_bits(bm))
@@ -92,6 +103,11 @@ class Session:
         side.synchronize()
         for a in self.adapter_ids:
             fl.fl_lora_register(self.pool, a, int(self.wl.ranks[a]), self.mats, self.lora_tables[a])
+
+    def _filler(self, n):
+        if getattr(self, "_filler_bits", None) is None or len(self._filler_bits) < n:
+            self._filler_bits = synth.bf16_bits(synth.Stream(self.wl.seed, "filler").normal((max(n, 1 << 20),), self.wl.weight_std))
+        return self._filler_bits[:n]
 
     # ---- batch index arrays and KV tables
     def build_batch(self):

@@ -7,6 +7,7 @@
 // shared memory with 16-byte cp.async through the block table and run QK^T and PV on bf16 tensor
 // cores with an fp32 online softmax.
 #include <math.h>
+#include <algorithm>
 #include "mma_utils.cuh"
 #include "attention.cuh"
 #include "pool.cuh"
@@ -72,6 +73,7 @@ __global__ void __launch_bounds__(256) attn_plan_kernel(const AttnArgs a, int ch
     a.hdr->n_prefill = min(base_p, a.max_prefill);
     a.hdr->n_decode = min(base_d, a.max_decode);
     a.hdr->chunk = chunk;
+    a.hdr->next_unit = 0;
   }
 }
 
@@ -524,7 +526,12 @@ int fl_paged_attention(fl_pool* p, fl_bf16* out, const fl_bf16* q, const int32_t
     const int kind = sm_scale > 0.f ? p->prefill_kernel : 1;
     attn_plan_kernel<<<1, 256, 0, st>>>(a, w.chunk, kind == 0 ? tc2_tile_tokens(n_q_heads, n_kv_heads) : (kind == 2 ? QT_TC : QT_MMA));
     if (kind == 0) {
-      rc = launch_prefill_tc2(p, a, n_tokens, w.max_prefill, st);
+      // upper bound of the plan's tile count: full tiles plus one ragged tile per prefill request, and a
+      // request is a prefill only with more than DEC_ROWS / group new tokens
+      const int group = n_q_heads / n_kv_heads;
+      const int max_req = std::min(n_req, n_tokens / (DEC_ROWS / group + 1));
+      const int max_items = std::min(w.max_prefill, n_tokens / tc2_tile_tokens(n_q_heads, n_kv_heads) + max_req);
+      rc = launch_prefill_tc2(p, a, n_tokens, max_items, st);
       if (rc != FL_OK) break;
     } else if (kind == 2) {
       rc = launch_prefill_tc(p, a, n_tokens, st);

@@ -16,7 +16,8 @@ constexpr int ATT_THREADS = 128;
 constexpr int DEC_ROWS = 16;
 
 struct PlanHdr {
-  int n_prefill, n_decode, chunk, pad;
+  int n_prefill, n_decode, chunk;
+  int next_unit;   // work counter of the persistent prefill kernel, zeroed by the plan kernel
 };
 
 struct AttnArgs {

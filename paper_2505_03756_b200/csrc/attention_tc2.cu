@@ -1,11 +1,12 @@
-// Prefill attention, two query tiles per CTA sharing one K/V stream (Section 2.1 / 4.2: attention over
-// the reused prefix KV plus the new tokens, read in place from pool blocks).
+// Prefill attention, two query tiles per CTA sharing one K/V stream, persistent CTAs (Section 2.1 / 4.2:
+// attention over the reused prefix KV plus the new tokens, read in place from pool blocks).
 //
-// One CTA per SM works on 2 x 128 query rows of one (request, KV head): with grouped heads the two
+// One CTA per SM.  A work unit is 2 x 128 query rows of one (request, KV head): with grouped heads the two
 // tiles are two query heads over the same 128 new tokens, otherwise two consecutive 128-token tiles of
 // one head.  Both tiles read the same K/V tiles, so every pool page is staged into shared memory once
-// for 256 query rows.
-//   warps 0-3   softmax of tile A (thread = query row = TMEM lane)      warp 8   TMA producer
+// for 256 query rows.  CTAs take units from a counter in device memory until none is left; the loads of
+// the next unit start while the current one is still in its last tiles and its epilogue.
+//   warps 0-3   softmax of tile A (thread = query row = TMEM lane)      warp 8   TMA producer, unit fetch
 //   warps 4-7   softmax of tile B                                        warp 9   MMA issuer, TMEM owner
 //   (warps 10, 11 only complete the third warpgroup, whose registers go to the softmax warpgroups)
 //   K_j / V_j (128 keys = 8 pool pages each) -> ring of 32 KiB slots, 128-byte swizzle
@@ -14,12 +15,14 @@
 //   O_X += P_X V_j      tcgen05.mma with the A operand read from TMEM, V MN-major as stored
 // The issuer alternates the tiles (PV_A, S_A, PV_B, S_B): while one tile's softmax runs, the tensor pipe
 // works for the other.  MMAs of one thread execute in issue order, so S_X(j+1) may overwrite P_X(j)
-// without a barrier, and "S_X(j+1) complete" implies "PV_X(j) complete".  O is rescaled only when a row
-// maximum grew by more than 2^8.  Every mbarrier wait is bounded; a wait that gives up raises a sticky
-// flag, the CTA drains its copies and frees its TMEM.
+// without a barrier, "S_X(j+1) complete" implies "PV_X(j) complete", and the first PV of a unit cannot
+// start before every softmax warp has finished the previous unit's epilogue (it waits for their P).
+// O is rescaled only when a row maximum grew by more than 2^8.  Every mbarrier wait is bounded; a wait
+// that gives up raises a sticky flag, the CTA drains its copies and frees its TMEM.
 #include <cuda.h>
 #include <math.h>
 #include <string.h>
+#include <algorithm>
 #include "attention.cuh"
 #include "mma_utils.cuh"
 #include "tc_ptx.cuh"
@@ -29,9 +32,9 @@ namespace {
 
 using namespace tc;
 
-constexpr int T2_THREADS = 384;                      // three warpgroups: softmax A, softmax B, {TMA, MMA, 2 idle warps}
+constexpr int T2_THREADS = 384;                        // three warpgroups: softmax A, softmax B, {TMA, MMA, 2 idle warps}
 constexpr int KT2 = 128;                               // keys per tile
-constexpr int NSLOT = 5;                               // ring slots; fills go K_0, V_0, K_1, V_1, ...
+constexpr int NSLOT = 5;                               // ring slots; fills go K_0, V_0, K_1, V_1, ... across units
 constexpr uint32_t HALF_BYTES = 128 * 128;             // [128 rows][64 bf16], swizzled
 constexpr uint32_t TILE_BYTES = 2 * HALF_BYTES;        // a Q, K or V tile
 constexpr uint32_t OFF_Q2 = 0;                         // Q_A, Q_B
@@ -40,71 +43,73 @@ constexpr uint32_t OFF_BAR2 = OFF_RING + NSLOT * TILE_BYTES;
 constexpr uint32_t T2_SMEM = OFF_BAR2 + 256;
 constexpr uint32_t T2_TMEM_COLS = 512;                 // S_A | S_B | O_A | O_B, 128 columns each
 constexpr float RESCALE_LOG2 = 8.f;
-#ifndef FL_POLY_OF_4
-#define FL_POLY_OF_4 0
-#endif
-constexpr int POLY_OF_4 = FL_POLY_OF_4;
 
-enum { C_QFULL = 0, C_FULL = 1, C_EMPTY = C_FULL + NSLOT, C_SFULL = C_EMPTY + NSLOT, C_PFULL = C_SFULL + 2,
-       C_ODONE = C_PFULL + 2, C_COUNT = C_ODONE + 2 };
+enum { C_QFULL = 0, C_QEMPTY = 1, C_FULL = 2, C_EMPTY = C_FULL + NSLOT, C_SFULL = C_EMPTY + NSLOT, C_PFULL = C_SFULL + 2,
+       C_ODONE = C_PFULL + 2, C_UFULL = C_ODONE + 2, C_UEMPTY = C_UFULL + 2, C_COUNT = C_UEMPTY + 2 };
+constexpr int UNIT_READERS = 9;                        // MMA issuer + 8 softmax warps
 
-struct Tile2 {          // what one CTA works on
+struct Unit {           // what a CTA works on at one time
   int tok0[2];          // first token row (in the packed q / out tensors) of each tile
   int hq[2];            // query head of each tile
   int rows[2];          // valid query rows (0 = tile unused)
   int lim0[2];          // last visible key of row 0 of each tile
   int n_kt[2];          // K/V tiles each tile takes part in
+  int n_kt_max, n_pages, tbl0, h;
+  bool valid;
 };
 
-__global__ void __launch_bounds__(T2_THREADS, 1)
-attn_prefill_tc2_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap kv_map, const __grid_constant__ CUtensorMap q_map,
-                        int heads_per_item) {
-  extern __shared__ __align__(1024) unsigned char smem[];
-  const int item = blockIdx.x / heads_per_item, hslot = blockIdx.x % heads_per_item;
-  if (item >= a.hdr->n_prefill) return;
-  const uint32_t sbase = smem_u32(smem);
-  if (sbase & 1023u) {   // the swizzled operand tiles need 1024-byte alignment
-    if (threadIdx.x == 0) atomicOr(a.pv.flags, (uint32_t)FLAG_WAIT_GAVE_UP);
-    return;
-  }
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+// Unit u = (plan tile u / heads_per_item, head slot u % heads_per_item).  Every role decodes it by itself.
+__device__ __forceinline__ Unit decode_unit(const AttnArgs& a, int u, int heads_per_item) {
+  Unit t;
+  const int item = u / heads_per_item, hslot = u % heads_per_item;
   const int2 it = a.prefill_list[item];
   const int i = it.x, q0 = it.y;
   const int n_new = a.new_lens[i], prefix = a.prefix_lens[i], ctx = prefix + n_new;
   const int group = a.n_q / a.n_kv;
-  const bool pair_heads = group % 2 == 0;
-  Tile2 t;
-  int h;   // KV head
-  if (pair_heads) {
+  if (group % 2 == 0) {
     t.hq[0] = 2 * hslot; t.hq[1] = 2 * hslot + 1;
-    h = t.hq[0] / group;
+    t.h = t.hq[0] / group;
     t.tok0[0] = t.tok0[1] = a.req_indptr[i] + q0;
     t.rows[0] = t.rows[1] = min(128, n_new - q0);
     t.lim0[0] = t.lim0[1] = prefix + q0;
   } else {
     t.hq[0] = t.hq[1] = hslot;
-    h = hslot / group;
+    t.h = hslot / group;
     t.tok0[0] = a.req_indptr[i] + q0; t.tok0[1] = t.tok0[0] + 128;
     t.rows[0] = min(128, n_new - q0); t.rows[1] = max(0, min(128, n_new - q0 - 128));
     t.lim0[0] = prefix + q0; t.lim0[1] = prefix + q0 + 128;
   }
 #pragma unroll
   for (int x = 0; x < 2; ++x) t.n_kt[x] = t.rows[x] > 0 ? (t.lim0[x] + t.rows[x] + KT2 - 1) / KT2 : 0;
-  const int n_kt = max(t.n_kt[0], t.n_kt[1]);
-  const int kv_end = min(ctx, n_kt * KT2);
-  const int tbl0 = a.tbl_indptr[i], tbl_n = a.tbl_indptr[i + 1] - tbl0;
-  const int n_pages = (kv_end + BT - 1) / BT;
-  if (n_pages > tbl_n || n_pages < 1 || t.rows[0] < 1) {
-    if (tid == 0) atomicOr(a.pv.flags, (uint32_t)FLAG_BAD_POS);
+  t.n_kt_max = max(t.n_kt[0], t.n_kt[1]);
+  const int kv_end = min(ctx, t.n_kt_max * KT2);
+  t.tbl0 = a.tbl_indptr[i];
+  t.n_pages = (kv_end + BT - 1) / BT;
+  t.valid = t.rows[0] >= 1 && t.n_pages >= 1 && t.n_pages <= a.tbl_indptr[i + 1] - t.tbl0;
+  return t;
+}
+
+__global__ void __launch_bounds__(T2_THREADS, 1)
+attn_prefill_tc2_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap kv_map, const __grid_constant__ CUtensorMap q_map,
+                        int heads_per_item) {
+  extern __shared__ __align__(1024) unsigned char smem[];
+  const int n_units = a.hdr->n_prefill * heads_per_item;
+  if ((int)blockIdx.x >= n_units) return;
+  const uint32_t sbase = smem_u32(smem);
+  if (sbase & 1023u) {   // the swizzled operand tiles need 1024-byte alignment
+    if (threadIdx.x == 0) atomicOr(a.pv.flags, (uint32_t)FLAG_WAIT_GAVE_UP);
     return;
   }
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const uint32_t bar0 = sbase + OFF_BAR2;
   auto bar = [&](int k) { return bar0 + 8u * k; };
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + OFF_BAR2 + 8 * C_COUNT);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + OFF_BAR2 + 8 * C_COUNT + 4);
+  volatile int* unit_slot = reinterpret_cast<volatile int*>(smem + OFF_BAR2 + 8 * C_COUNT + 8);   // [2]
 
   if (tid == 0) {
     mbar_init(bar(C_QFULL), 1);
+    mbar_init(bar(C_QEMPTY), 1);
     for (int s = 0; s < NSLOT; ++s) {
       mbar_init(bar(C_FULL + s), 1);
       mbar_init(bar(C_EMPTY + s), 1);
@@ -113,6 +118,8 @@ attn_prefill_tc2_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap kv
       mbar_init(bar(C_SFULL + x), 1);
       mbar_init(bar(C_PFULL + x), 4);
       mbar_init(bar(C_ODONE + x), 1);
+      mbar_init(bar(C_UFULL + x), 1);
+      mbar_init(bar(C_UEMPTY + x), UNIT_READERS);
     }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -126,53 +133,80 @@ attn_prefill_tc2_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap kv
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
 
+  // Readers take the k-th unit of this CTA from slot k & 1 (-1 = no more work) and release the slot.
+  auto read_unit = [&](int k, bool arrive) -> int {
+    if (!mbar_wait(bar(C_UFULL + (k & 1)), (k >> 1) & 1, abort_flag)) return -1;
+    const int u = unit_slot[k & 1];
+    if (arrive) mbar_arrive(bar(C_UEMPTY + (k & 1)));
+    return u;
+  };
+
   // the softmax warpgroups keep 128 scores per thread in registers: they take the registers the third
   // warpgroup does not need
   if (warp >= 8) {
-  asm volatile("setmaxnreg.dec.sync.aligned.u32 40;");
-  if (warp == 8) {
-    // ------------------------------------------------ TMA producer
-    if (lane == 0) {
-      mbar_expect_tx(bar(C_QFULL), t.rows[1] > 0 ? 2 * TILE_BYTES : TILE_BYTES);
-#pragma unroll
-      for (int x = 0; x < 2; ++x) {
-        if (t.rows[x] > 0) {
-          tma_load_3d(sbase + OFF_Q2 + x * TILE_BYTES, &q_map, bar(C_QFULL), 0, t.hq[x], t.tok0[x]);
-          tma_load_3d(sbase + OFF_Q2 + x * TILE_BYTES + HALF_BYTES, &q_map, bar(C_QFULL), 64, t.hq[x], t.tok0[x]);
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
+    if (warp == 8 && lane == 0) {
+      // ------------------------------------------------ unit fetch + TMA producer
+      int fill = 0;                    // ring fills so far, over all units
+      int n_valid = 0;                 // units whose Q tiles were loaded so far
+      for (int k = 0;; ++k) {
+        if (k >= 2 && !mbar_wait(bar(C_UEMPTY + (k & 1)), ((k >> 1) - 1) & 1, abort_flag)) break;
+        int u = k == 0 ? (int)blockIdx.x : (int)gridDim.x + atomicAdd(&a.hdr->next_unit, 1);
+        if (u >= n_units) u = -1;
+        unit_slot[k & 1] = u;
+        mbar_arrive(bar(C_UFULL + (k & 1)));
+        if (u < 0) break;
+        const Unit t = decode_unit(a, u, heads_per_item);
+        if (!t.valid) {
+          atomicOr(a.pv.flags, (uint32_t)FLAG_BAD_POS);
+          continue;
         }
-      }
-      bool ok = true;
-      for (int idx = 0; ok && idx < 2 * n_kt; ++idx) {
-        const int j = idx >> 1, side = idx & 1;
-        const int s = idx % NSLOT, use = idx / NSLOT;
-        if (use > 0 && !mbar_wait(bar(C_EMPTY + s), (use - 1) & 1, abort_flag)) break;
-        mbar_expect_tx(bar(C_FULL + s), TILE_BYTES);
-        const uint32_t dst = sbase + OFF_RING + s * TILE_BYTES;
-        const int slot_head = side * a.n_kv + h;
+        // Q buffers are free once the previous unit's last S MMA has completed
+        if (n_valid > 0 && !mbar_wait(bar(C_QEMPTY), (n_valid - 1) & 1, abort_flag)) break;
+        ++n_valid;
+        mbar_expect_tx(bar(C_QFULL), t.rows[1] > 0 ? 2 * TILE_BYTES : TILE_BYTES);
 #pragma unroll
-        for (int pg = 0; pg < KT2 / BT; ++pg) {
-          // pages behind the last needed key are masked anyway: re-read the last valid page
-          const int page = min(j * (KT2 / BT) + pg, n_pages - 1);
-          uint32_t blk = a.tbl[tbl0 + page];
-          if (blk >= a.pv.n_blocks) {
-            atomicOr(a.pv.flags, (uint32_t)FLAG_BAD_BLOCK);
-            blk = 0;
+        for (int x = 0; x < 2; ++x) {
+          if (t.rows[x] > 0) {
+            tma_load_3d(sbase + OFF_Q2 + x * TILE_BYTES, &q_map, bar(C_QFULL), 0, t.hq[x], t.tok0[x]);
+            tma_load_3d(sbase + OFF_Q2 + x * TILE_BYTES + HALF_BYTES, &q_map, bar(C_QFULL), 64, t.hq[x], t.tok0[x]);
           }
-          const uint32_t off = pg * (BT * 128);
-          tma_load_4d(dst + off, &kv_map, bar(C_FULL + s), 0, 0, slot_head, (int)blk);
-          tma_load_4d(dst + HALF_BYTES + off, &kv_map, bar(C_FULL + s), 64, 0, slot_head, (int)blk);
         }
+        bool ok = true;
+        for (int idx = 0; idx < 2 * t.n_kt_max; ++idx, ++fill) {
+          const int j = idx >> 1, side = idx & 1;
+          const int s = fill % NSLOT, use = fill / NSLOT;
+          if (use > 0 && !mbar_wait(bar(C_EMPTY + s), (use - 1) & 1, abort_flag)) { ok = false; break; }
+          mbar_expect_tx(bar(C_FULL + s), TILE_BYTES);
+          const uint32_t dst = sbase + OFF_RING + s * TILE_BYTES;
+          const int slot_head = side * a.n_kv + t.h;
+#pragma unroll
+          for (int pg = 0; pg < KT2 / BT; ++pg) {
+            // pages behind the last needed key are masked anyway: re-read the last valid page
+            const int page = min(j * (KT2 / BT) + pg, t.n_pages - 1);
+            uint32_t blk = a.tbl[t.tbl0 + page];
+            if (blk >= a.pv.n_blocks) {
+              atomicOr(a.pv.flags, (uint32_t)FLAG_BAD_BLOCK);
+              blk = 0;
+            }
+            const uint32_t off = pg * (BT * 128);
+            tma_load_4d(dst + off, &kv_map, bar(C_FULL + s), 0, 0, slot_head, (int)blk);
+            tma_load_4d(dst + HALF_BYTES + off, &kv_map, bar(C_FULL + s), 64, 0, slot_head, (int)blk);
+          }
+        }
+        if (!ok) break;
       }
-    }
-  } else if (warp == 9) {
-    // ------------------------------------------------ MMA issuer
-    if (lane == 0) {
+    } else if (warp == 9 && lane == 0) {
+      // ------------------------------------------------ MMA issuer
       constexpr uint32_t IDESC = instr_desc(128, false);        // S: both operands K-major
       constexpr uint32_t IDESC_PV = instr_desc(D, true);        // O: V is MN-major
+      int cons = 0;                    // ring slots consumed so far, over all units
+      int steps[2] = {0, 0};           // P tiles awaited so far per tile (phase of C_PFULL)
+      int n_done = 0;                  // valid units so far (phase of C_QFULL)
       auto slot_addr = [&](int idx) { return sbase + OFF_RING + (idx % NSLOT) * TILE_BYTES; };
       auto wait_full = [&](int idx) { return mbar_wait(bar(C_FULL + idx % NSLOT), (idx / NSLOT) & 1, abort_flag); };
-      auto issue_s = [&](int x, int j) {
-        const uint32_t qb = sbase + OFF_Q2 + x * TILE_BYTES, kb = slot_addr(2 * j);
+      auto issue_s = [&](int x, int kslot) {
+        const uint32_t qb = sbase + OFF_Q2 + x * TILE_BYTES, kb = slot_addr(kslot);
 #pragma unroll
         for (int ks = 0; ks < D / 16; ++ks) {
           const uint32_t off = (ks >> 2) * HALF_BYTES + (ks & 3) * 32;
@@ -180,162 +214,168 @@ attn_prefill_tc2_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap kv
         }
         umma_commit(bar(C_SFULL + x));
       };
-      auto issue_pv = [&](int x, int j, bool last) {
-        const uint32_t vb = slot_addr(2 * j + 1);
+      auto issue_pv = [&](int x, int vslot, bool first, bool last) {
+        const uint32_t vb = slot_addr(vslot);
 #pragma unroll
         for (int ks = 0; ks < KT2 / 16; ++ks)
           umma_bf16_ts(tmem + 256 + x * 128, tmem + x * 128 + ks * 8, smem_desc(vb + ks * (16 * 128), HALF_BYTES, 1024),
-                       IDESC_PV, (j > 0 || ks > 0));
+                       IDESC_PV, (!first || ks > 0));
         if (last) umma_commit(bar(C_ODONE + x));
       };
-      bool ok = mbar_wait(bar(C_QFULL), 0, abort_flag) && wait_full(0);
-      if (ok) {
-        tc_fence_after();
-        if (t.n_kt[0] > 0) issue_s(0, 0);
-        if (t.n_kt[1] > 0) issue_s(1, 0);
-        umma_commit(bar(C_EMPTY + 0));
-      }
-      for (int j = 0; ok && j < n_kt; ++j) {
-        const bool more = j + 1 < n_kt;
-        ok = wait_full(2 * j + 1);
-        if (ok && j < t.n_kt[0]) {
-          ok = mbar_wait(bar(C_PFULL + 0), j & 1, abort_flag);
-          if (ok) { tc_fence_after(); issue_pv(0, j, j == t.n_kt[0] - 1); }
-        }
-        if (ok && more) ok = wait_full(2 * j + 2);
+      bool ok = true;
+      for (int k = 0; ok; ++k) {
+        const int u = read_unit(k, true);
+        if (u < 0) break;
+        const Unit t = decode_unit(a, u, heads_per_item);
+        if (!t.valid) continue;
+        const int n_kt = t.n_kt_max, nA = t.n_kt[0], nB = t.n_kt[1];
+        const int base = cons;         // ring index of K_0 of this unit; K_j = base + 2j, V_j = base + 2j + 1
+        ok = mbar_wait(bar(C_QFULL), n_done & 1, abort_flag) && wait_full(base);
         if (!ok) break;
+        ++n_done;
         tc_fence_after();
-        if (j + 1 < t.n_kt[0]) issue_s(0, j + 1);
-        if (j < t.n_kt[1]) {
-          ok = mbar_wait(bar(C_PFULL + 1), j & 1, abort_flag);
+        if (nA > 0) issue_s(0, base);
+        if (nB > 0) issue_s(1, base);
+        umma_commit(bar(C_EMPTY + base % NSLOT));
+        if (n_kt == 1) umma_commit(bar(C_QEMPTY));
+        for (int j = 0; ok && j < n_kt; ++j) {
+          const bool more = j + 1 < n_kt;
+          const int vs = base + 2 * j + 1, kn = base + 2 * j + 2;
+          ok = wait_full(vs);
+          if (ok && j < nA) {
+            ok = mbar_wait(bar(C_PFULL + 0), steps[0]++ & 1, abort_flag);
+            if (ok) { tc_fence_after(); issue_pv(0, vs, j == 0, j == nA - 1); }
+          }
+          if (ok && more) ok = wait_full(kn);
           if (!ok) break;
           tc_fence_after();
-          issue_pv(1, j, j == t.n_kt[1] - 1);
+          if (j + 1 < nA) issue_s(0, kn);
+          if (j < nB) {
+            ok = mbar_wait(bar(C_PFULL + 1), steps[1]++ & 1, abort_flag);
+            if (!ok) break;
+            tc_fence_after();
+            issue_pv(1, vs, j == 0, j == nB - 1);
+          }
+          umma_commit(bar(C_EMPTY + vs % NSLOT));
+          if (j + 1 < nB) issue_s(1, kn);
+          if (more) umma_commit(bar(C_EMPTY + kn % NSLOT));
+          if (j + 2 == n_kt) umma_commit(bar(C_QEMPTY));     // the unit's last S MMAs are in the pipe: Q is free after them
         }
-        umma_commit(bar(C_EMPTY + (2 * j + 1) % NSLOT));
-        if (j + 1 < t.n_kt[1]) issue_s(1, j + 1);
-        if (more) umma_commit(bar(C_EMPTY + (2 * j + 2) % NSLOT));
+        cons = base + 2 * n_kt;
       }
     }
-  }
   } else {
-    asm volatile("setmaxnreg.inc.sync.aligned.u32 232;");
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
     // ------------------------------------------------ softmax of tile x: thread = query row = TMEM lane
     const int x = warp >> 2, row = tid & 127;
-    const int rows = x ? t.rows[1] : t.rows[0], nk = x ? t.n_kt[1] : t.n_kt[0];
-    const int lim = row < rows ? (x ? t.lim0[1] : t.lim0[0]) + row : -1;
-    const int out_tok0 = x ? t.tok0[1] : t.tok0[0], out_hq = x ? t.hq[1] : t.hq[0];
     const uint32_t lane_addr = tmem + ((uint32_t)((warp & 3) * 32) << 16);
     const uint32_t s_addr = lane_addr + x * 128, o_addr = lane_addr + 256 + x * 128;
     const float sl2 = a.scale_log2;
-    float m_used = 0.f, m_run = -INFINITY, l = 0.f;
-    bool ok = nk > 0;
-    for (int j = 0; j < nk; ++j) {
-      ok = mbar_wait(bar(C_SFULL + x), j & 1, abort_flag);
-      if (!ok) break;
-      tc_fence_after();
-      uint32_t s[4][32];
+    int steps = 0;      // S tiles of this tile taken so far (phase of C_SFULL)
+    int epis = 0;       // epilogues so far (phase of C_ODONE)
+    for (int k = 0;; ++k) {
+      const int u = read_unit(k, false);
+      __syncwarp();
+      if (lane == 0 && u >= 0) mbar_arrive(bar(C_UEMPTY + (k & 1)));
+      if (u < 0) break;
+      const Unit t = decode_unit(a, u, heads_per_item);
+      if (!t.valid) continue;
+      const int rows = x ? t.rows[1] : t.rows[0], nk = x ? t.n_kt[1] : t.n_kt[0];
+      if (nk == 0) continue;
+      const int lim = row < rows ? (x ? t.lim0[1] : t.lim0[0]) + row : -1;
+      float m_used = 0.f, m_run = -INFINITY, l = 0.f;
+      bool ok = true;
+      for (int j = 0; j < nk; ++j) {
+        ok = mbar_wait(bar(C_SFULL + x), steps++ & 1, abort_flag);
+        if (!ok) break;
+        tc_fence_after();
+        uint32_t s[4][32];
 #pragma unroll
-      for (int c = 0; c < 4; ++c) tmem_ld32(s_addr + 32 * c, s[c]);
-      tmem_wait_ld();
-      const int u0 = j * KT2;
-      if (u0 + KT2 - 1 > lim) {     // a tile that reaches past this row's last visible key
+        for (int c = 0; c < 4; ++c) tmem_ld32(s_addr + 32 * c, s[c]);
+        tmem_wait_ld();
+        const int u0 = j * KT2;
+        if (u0 + KT2 - 1 > lim) {     // a tile that reaches past this row's last visible key
+#pragma unroll
+          for (int c = 0; c < 4; ++c)
+#pragma unroll
+            for (int e = 0; e < 32; ++e)
+              if (u0 + 32 * c + e > lim) s[c][e] = 0xff800000u;   // -inf
+        }
+        float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
         for (int c = 0; c < 4; ++c)
 #pragma unroll
-          for (int e = 0; e < 32; ++e)
-            if (u0 + 32 * c + e > lim) s[c][e] = 0xff800000u;   // -inf
-      }
-      float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-#pragma unroll
-      for (int c = 0; c < 4; ++c)
-#pragma unroll
-        for (int e = 0; e < 32; e += 2)
-          mx[(e >> 1) & 3] = max3(mx[(e >> 1) & 3], __uint_as_float(s[c][e]), __uint_as_float(s[c][e + 1]));
-      m_run = fmaxf(m_run, fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])));
-      bool rescale = false;
-      float alpha = 1.f;
-      if (j == 0) {
-        m_used = m_run == -INFINITY ? 0.f : m_run;
-      } else if ((m_run - m_used) * sl2 > RESCALE_LOG2) {
-        rescale = true;
-        alpha = ex2_approx((m_used - m_run) * sl2);
-        m_used = m_run;
-      }
-      // S_X(j) complete implies PV_X(j-1) complete: O may be touched here
-      if (__any_sync(0xffffffffu, rescale)) {
-#pragma unroll
-        for (int cb = 0; cb < D; cb += 32) {
-          uint32_t o[32];
-          tmem_ld32(o_addr + cb, o);
-          tmem_wait_ld();
-#pragma unroll
-          for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * alpha);
-          tmem_st32(o_addr + cb, o);
+          for (int e = 0; e < 32; e += 2)
+            mx[(e >> 1) & 3] = max3(mx[(e >> 1) & 3], __uint_as_float(s[c][e]), __uint_as_float(s[c][e + 1]));
+        m_run = fmaxf(m_run, fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])));
+        bool rescale = false;
+        float alpha = 1.f;
+        if (j == 0) {
+          m_used = m_run == -INFINITY ? 0.f : m_run;
+        } else if ((m_run - m_used) * sl2 > RESCALE_LOG2) {
+          rescale = true;
+          alpha = ex2_approx((m_used - m_run) * sl2);
+          m_used = m_run;
         }
-        l *= alpha;
-      }
-      const float2 sc2 = make_float2(sl2, sl2);
-      const float nm = -m_used * sl2;
-      const float2 nm2 = make_float2(nm, nm);
-      float2 sum[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+        // S_X(j) complete implies PV_X(j-1) complete: O may be touched here
+        if (__any_sync(0xffffffffu, rescale)) {
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {      // 32 keys -> 16 bf16 pairs -> TMEM columns 16c .. 16c+15 of this tile
-        uint32_t pk[16];
+          for (int cb = 0; cb < D; cb += 32) {
+            uint32_t o[32];
+            tmem_ld32(o_addr + cb, o);
+            tmem_wait_ld();
 #pragma unroll
-        for (int e = 0; e < 16; ++e) {
-          const float2 arg = __ffma2_rn(make_float2(__uint_as_float(s[c][2 * e]), __uint_as_float(s[c][2 * e + 1])), sc2, nm2);
-          // POLY_OF_4 of every 4 pairs take the polynomial, the others the special-function unit: the two
-          // run side by side and the slower unit no longer sets the pace of the tile
-          const float2 p = (e & 3) < POLY_OF_4 ? ex2_poly2(arg) : make_float2(ex2_approx(arg.x), ex2_approx(arg.y));
-          sum[e & 1] = __fadd2_rn(sum[e & 1], p);
-          pk[e] = pack_bf16(p.x, p.y);
+            for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * alpha);
+            tmem_st32(o_addr + cb, o);
+          }
+          l *= alpha;
         }
-        tmem_st16(s_addr + 16 * c, pk);
+        const float2 sc2 = make_float2(sl2, sl2);
+        const float nm = -m_used * sl2;
+        const float2 nm2 = make_float2(nm, nm);
+        float2 sum[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {      // 32 keys -> 16 bf16 pairs -> TMEM columns 16c .. 16c+15 of this tile
+          uint32_t pk[16];
+#pragma unroll
+          for (int e = 0; e < 16; ++e) {
+            const float2 arg = __ffma2_rn(make_float2(__uint_as_float(s[c][2 * e]), __uint_as_float(s[c][2 * e + 1])), sc2, nm2);
+            const float2 p = make_float2(ex2_approx(arg.x), ex2_approx(arg.y));
+            sum[e & 1] = __fadd2_rn(sum[e & 1], p);
+            pk[e] = pack_bf16(p.x, p.y);
+          }
+          tmem_st16(s_addr + 16 * c, pk);
+        }
+        l += (sum[0].x + sum[0].y) + (sum[1].x + sum[1].y);
+        tmem_wait_st();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar(C_PFULL + x));
       }
-      l += (sum[0].x + sum[0].y) + (sum[1].x + sum[1].y);
-      tmem_wait_st();
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bar(C_PFULL + x));
-    }
-    // ---- epilogue: O / l -> bf16 -> staged in this tile's Q buffer -> coalesced 16-byte stores
-    if (ok) ok = mbar_wait(bar(C_ODONE + x), 0, abort_flag);
-    unsigned char* stage = smem + OFF_Q2 + x * TILE_BYTES;
-    if (ok) {
+      // ---- epilogue: O / l -> bf16, each thread stores its own row (16 x 16 bytes, contiguous)
+      if (ok) ok = mbar_wait(bar(C_ODONE + x), epis++ & 1, abort_flag);
+      if (!ok) break;
       tc_fence_after();
       const float inv = l > 0.f ? 1.f / l : 0.f;
-      unsigned char* orow = stage + row * 256;
+      uint4* orow = reinterpret_cast<uint4*>(a.out + ((size_t)((x ? t.tok0[1] : t.tok0[0]) + row) * a.n_q + (x ? t.hq[1] : t.hq[0])) * D);
 #pragma unroll
       for (int cb = 0; cb < D; cb += 32) {
         uint32_t o[32];
         tmem_ld32(o_addr + cb, o);
         tmem_wait_ld();
+        if (row < rows) {
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          uint4 v;
-          v.x = pack_bf16(__uint_as_float(o[8 * c + 0]) * inv, __uint_as_float(o[8 * c + 1]) * inv);
-          v.y = pack_bf16(__uint_as_float(o[8 * c + 2]) * inv, __uint_as_float(o[8 * c + 3]) * inv);
-          v.z = pack_bf16(__uint_as_float(o[8 * c + 4]) * inv, __uint_as_float(o[8 * c + 5]) * inv);
-          v.w = pack_bf16(__uint_as_float(o[8 * c + 6]) * inv, __uint_as_float(o[8 * c + 7]) * inv);
-          const int chunk = (cb >> 3) + c;
-          *reinterpret_cast<uint4*>(orow + ((chunk ^ (row & 7)) << 4)) = v;
+          for (int c = 0; c < 4; ++c) {
+            uint4 v;
+            v.x = pack_bf16(__uint_as_float(o[8 * c + 0]) * inv, __uint_as_float(o[8 * c + 1]) * inv);
+            v.y = pack_bf16(__uint_as_float(o[8 * c + 2]) * inv, __uint_as_float(o[8 * c + 3]) * inv);
+            v.z = pack_bf16(__uint_as_float(o[8 * c + 4]) * inv, __uint_as_float(o[8 * c + 5]) * inv);
+            v.w = pack_bf16(__uint_as_float(o[8 * c + 6]) * inv, __uint_as_float(o[8 * c + 7]) * inv);
+            orow[(cb >> 3) + c] = v;
+          }
         }
       }
       tc_fence_before();
-    }
-    // the four warps of a tile exchange rows through shared memory: named barrier over its 128 threads
-    if (x == 0) asm volatile("bar.sync 1, 128;" ::: "memory");
-    else asm volatile("bar.sync 2, 128;" ::: "memory");
-    if (ok && !*abort_flag) {
-      const int cch = row & 15;
-#pragma unroll
-      for (int r = 0; r < 16; ++r) {
-        const int orow_i = (row >> 4) + 8 * r;
-        if (orow_i < rows)
-          *reinterpret_cast<uint4*>(a.out + ((size_t)(out_tok0 + orow_i) * a.n_q + out_hq) * D + cch * 8) =
-              *reinterpret_cast<const uint4*>(stage + orow_i * 256 + ((cch ^ (orow_i & 7)) << 4));
-      }
     }
   }
   // ------------------------------------------------ teardown
@@ -349,6 +389,8 @@ attn_prefill_tc2_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap kv
       for (int s = 0; s < NSLOT; ++s)
         for (uint32_t k = 0; k < (1u << 16); ++k)
           if (mbar_try(bar(C_FULL + s), 0) || mbar_try(bar(C_FULL + s), 1)) break;
+      for (uint32_t k = 0; k < (1u << 16); ++k)
+        if (mbar_try(bar(C_QFULL), 0) || mbar_try(bar(C_QFULL), 1)) break;
     }
     __syncthreads();
   }
@@ -372,7 +414,11 @@ int launch_prefill_tc2(fl_pool* p, const AttnArgs& a, int n_tokens, int max_item
   }
   const int group = a.n_q / a.n_kv;
   const int heads_per_item = group % 2 == 0 ? a.n_q / 2 : a.n_q;
-  attn_prefill_tc2_kernel<<<(unsigned)max_items * heads_per_item, T2_THREADS, T2_SMEM, st>>>(a, *kv, qmap, heads_per_item);
+  // one CTA per SM (shared memory and TMEM allow no more); CTAs beyond the plan's unit count exit at once
+  const long long units = (long long)max_items * heads_per_item;
+  const unsigned grid = (unsigned)std::min<long long>(units, p->sm_count);
+  if (grid == 0) return FL_OK;
+  attn_prefill_tc2_kernel<<<grid, T2_THREADS, T2_SMEM, st>>>(a, *kv, qmap, heads_per_item);
   FL_CUDA(p, cudaGetLastError());
   return FL_OK;
 }

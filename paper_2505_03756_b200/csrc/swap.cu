@@ -148,11 +148,26 @@ __global__ void kv_append_kernel(PoolView pv, const uint4* __restrict__ k_new, c
   constexpr int CH = FL_HEAD_DIM * 2 / 16;                     // 16-byte chunks per (head, token) row
   uint4* dst = reinterpret_cast<uint4*>(pv.slab + (size_t)blk * pv.block_bytes);
   const int per_side = n_kv * CH;
-  for (int c = threadIdx.x; c < 2 * per_side; c += blockDim.x) {
-    const int w = c / per_side, r = c - w * per_side;
-    const int h = r / CH, e = r - h * CH;
-    const uint4 val = (w ? v_new : k_new)[(size_t)t * per_side + r];
-    dst[((size_t)(w * n_kv + h) * bt + slot) * CH + e] = val;
+  // four independent 16-byte loads in flight per thread before the first store
+  for (int c0 = threadIdx.x; c0 < 2 * per_side; c0 += 4 * blockDim.x) {
+    uint4 val[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int c = c0 + u * blockDim.x;
+      if (c < 2 * per_side) {
+        const int w = c / per_side, r = c - w * per_side;
+        val[u] = (w ? v_new : k_new)[(size_t)t * per_side + r];
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int c = c0 + u * blockDim.x;
+      if (c < 2 * per_side) {
+        const int w = c / per_side, r = c - w * per_side;
+        const int h = r / CH, e = r - h * CH;
+        dst[((size_t)(w * n_kv + h) * bt + slot) * CH + e] = val[u];
+      }
+    }
   }
   // The request's last token also clears the V slots behind it in its block, so that attention can
   // multiply those slots by a zero weight without meeting stale non-finite bit patterns.

@@ -173,25 +173,35 @@ attn_prefill_tc2_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap kv
           }
         }
         bool ok = true;
-        for (int idx = 0; idx < 2 * t.n_kt_max; ++idx, ++fill) {
-          const int j = idx >> 1, side = idx & 1;
-          const int s = fill % NSLOT, use = fill / NSLOT;
-          if (use > 0 && !mbar_wait(bar(C_EMPTY + s), (use - 1) & 1, abort_flag)) { ok = false; break; }
-          mbar_expect_tx(bar(C_FULL + s), TILE_BYTES);
-          const uint32_t dst = sbase + OFF_RING + s * TILE_BYTES;
-          const int slot_head = side * a.n_kv + t.h;
+        for (int j = 0; ok && j < t.n_kt_max; ++j) {
+          // the tile's eight block ids first (independent loads, in flight together, before any wait); K_j and
+          // V_j come from the same blocks
+          uint32_t blk[KT2 / BT];
+#pragma unroll
+          for (int pg = 0; pg < KT2 / BT; ++pg)   // pages behind the last needed key are masked anyway: re-read the last valid page
+            blk[pg] = a.tbl[t.tbl0 + min(j * (KT2 / BT) + pg, t.n_pages - 1)];
+          bool bad = false;
 #pragma unroll
           for (int pg = 0; pg < KT2 / BT; ++pg) {
-            // pages behind the last needed key are masked anyway: re-read the last valid page
-            const int page = min(j * (KT2 / BT) + pg, t.n_pages - 1);
-            uint32_t blk = a.tbl[t.tbl0 + page];
-            if (blk >= a.pv.n_blocks) {
-              atomicOr(a.pv.flags, (uint32_t)FLAG_BAD_BLOCK);
-              blk = 0;
+            if (blk[pg] >= a.pv.n_blocks) {
+              bad = true;
+              blk[pg] = 0;
             }
-            const uint32_t off = pg * (BT * 128);
-            tma_load_4d(dst + off, &kv_map, bar(C_FULL + s), 0, 0, slot_head, (int)blk);
-            tma_load_4d(dst + HALF_BYTES + off, &kv_map, bar(C_FULL + s), 64, 0, slot_head, (int)blk);
+          }
+          if (bad) atomicOr(a.pv.flags, (uint32_t)FLAG_BAD_BLOCK);
+#pragma unroll
+          for (int side = 0; side < 2; ++side, ++fill) {
+            const int s = fill % NSLOT, use = fill / NSLOT;
+            if (use > 0 && !mbar_wait(bar(C_EMPTY + s), (use - 1) & 1, abort_flag)) { ok = false; break; }
+            mbar_expect_tx(bar(C_FULL + s), TILE_BYTES);
+            const uint32_t dst = sbase + OFF_RING + s * TILE_BYTES;
+            const int slot_head = side * a.n_kv + t.h;
+#pragma unroll
+            for (int pg = 0; pg < KT2 / BT; ++pg) {
+              const uint32_t off = pg * (BT * 128);
+              tma_load_4d(dst + off, &kv_map, bar(C_FULL + s), 0, 0, slot_head, (int)blk[pg]);
+              tma_load_4d(dst + HALF_BYTES + off, &kv_map, bar(C_FULL + s), 64, 0, slot_head, (int)blk[pg]);
+            }
           }
         }
         if (!ok) break;

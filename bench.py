@@ -223,6 +223,8 @@ def run_ours(args, wl):
     T = wl.n_tokens
     n_swap = args.swap_blocks if args.swap_blocks >= 0 else (256 if args.workload == "swapstress" else 32)
     sess = H.Session(wl, device=local, extra_host_blocks=2 * n_swap, register_all=(args.workload == "swapstress"))
+    if args.prefill_kernel >= 0:
+        fl.fl_pool_set_option(sess.pool, fl.FL_OPT_PREFILL_KERNEL, args.prefill_kernel)
     sess.load_adapters()
     # the new-token blocks are taken and returned every step (allocator on the path); tables stay put
     sess.build_batch()
@@ -429,6 +431,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="prefill7b", choices=list(WORKLOAD_TEXT))
     ap.add_argument("--swap-blocks", type=int, default=-1)
+    ap.add_argument("--prefill-kernel", type=int, default=-1, help="FL_OPT_PREFILL_KERNEL value (default: the library's)")
     ap.add_argument("--n-req", type=int, default=0, help="reduced copy of the workload with this many requests "
                     "(small pool; for profiler captures, not a bench line)")
     args = ap.parse_args()

@@ -31,6 +31,11 @@ WORKLOAD_TEXT = {
 }
 
 
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of a call's kernels, from the ncu captures summarised
+# under profiles/ (bytes); absent = not captured for the current kernels
+NCU_TRAFFIC = {("prefill7b", "attention"): 864.3e6}
+
+
 def peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
@@ -393,7 +398,8 @@ def run_ours(args, wl):
         else:
             ach, peak, unit = w["bytes"] / sec / 1e9, pk["hbm"], "GB/s"
         roof = {"kernel": top, "bound": w["bound"], "achieved": round(ach, 2), "peak": peak, "unit": unit,
-                "frac": round(ach / peak, 4), "traffic": None, "peak_source": pk["src"] + " (burst)",
+                "frac": round(ach / peak, 4), "traffic": NCU_TRAFFIC.get((args.workload, top)) if not args.n_req else None,
+                "algorithmic_bytes": int(w["bytes"]), "peak_source": pk["src"] + " (burst)",
                 "ms_per_launch": round(call_ms[top], 4)}
         cb, _, _ = oracle_baseline(wl)
         h2d = int(h_x.numel() * 2 + sum(h_y[m].numel() * 2 for m in names))

@@ -259,11 +259,12 @@ def run_ours(args, wl):
     # shrink + expand per SGMV call, KV append, plan + prefill + decode + merge, swap gather + scatter
     launches_per_step = 2 + 1 + 4 + 2 + (4 if s.inter else 0) + (2 * -(-n_swap // 256) if n_swap > 1 else 0)
 
-    def step(k, evs=None):
+    def step(k, evs=None, swap=True):
         sign = wl.scale if k % 2 == 0 else -wl.scale     # y += s*delta, then y -= s*delta: values stay bounded
         ids = fl.fl_block_alloc(sess.pool, spare)        # a1: the allocator runs every step
         fl.fl_block_free(sess.pool, ids[::-1])
-        if n_swap:                                        # a7: side stream, overlapped
+        swap = swap and n_swap > 0
+        if swap:                                          # a7: side streams, overlapped
             fl.fl_swap_out(sess.pool, swap_dev_out, swap_host_out, side)
             fl.fl_swap_in(sess.pool, swap_dev_in, swap_host_in, side_in)
         mark = (lambda: None) if evs is None else (lambda: evs.append(_rec(torch, main)))
@@ -281,7 +282,7 @@ def run_ours(args, wl):
             mark()
             sess.sgmv([d_y["down"]], d_y["up"], ["down"], scale=sign, stream=main)
             mark()
-        if n_swap:
+        if swap:
             ev_side.record(side)
             ev_side_in.record(side_in)
             main.wait_event(ev_side)
@@ -334,6 +335,17 @@ def run_ours(args, wl):
         f1.record(main)
         barrier()
         ms_e2e = f0.elapsed_time(f1) / e2e_steps
+        # the same steps without the concurrent swap: how much of the swap the kernels hide
+        overlap = None
+        if n_swap:
+            barrier()
+            h0, h1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            h0.record(main)
+            for k in range(args.steps):
+                step(k, swap=False)
+            h1.record(main)
+            barrier()
+            overlap = {"ms_per_step_without_swap": h0.elapsed_time(h1) / args.steps}
         # the swap alone (both directions at once), and the host link's own peak for the same byte count
         swap = None
         if n_swap:
@@ -391,6 +403,10 @@ def run_ours(args, wl):
             kernels[c] = k
         if swap:
             kernels["swap"] = swap
+            # 1 = the step with the swap costs no more than the longer of (step without swap, swap alone)
+            overlap["ms_per_step_with_swap"] = ms_step
+            overlap["efficiency"] = round(max(overlap["ms_per_step_without_swap"], swap["ms"]) / ms_step, 4)
+            overlap["ms_per_step_without_swap"] = round(overlap["ms_per_step_without_swap"], 4)
         top = max(calls, key=lambda c: call_ms[c])
         w, sec = wm[top], call_ms[top] * 1e-3
         if w["bound"] == "tensor":
@@ -412,7 +428,7 @@ def run_ours(args, wl):
                        "block_bytes": s.block_bytes, "swap_blocks_each_way": n_swap,
                        "l2": "inputs larger than L2 (x, y and KV exceed 126 MB); no flush between steps",
                        "parallelism": "independent batch per GPU, no collective"},
-            "roofline": roof, "kernels": kernels, "cpu_baseline": cb,
+            "roofline": roof, "kernels": kernels, "swap_overlap": overlap, "cpu_baseline": cb,
             "e2e": {"value": tokens_all / (ms_e2e * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": int(h_out.numel() * 2), "ms_per_step": ms_e2e},
             "gpu_launches": launches_per_step * args.steps, "clocks": clocks, "device_flags": flags,

@@ -218,6 +218,45 @@ int fl_swap_in(fl_pool* pool, const uint32_t* dev_ids, const uint32_t* host_ids,
 int fl_swap_record(fl_pool* pool, fl_event ev, fl_stream side);
 int fl_swap_wait(fl_pool* pool, fl_event ev, int timeout_ms);
 
+/* ---------------------------------------------------------------- cache swapper (Section 5; host code, no GPU work)
+ * Decides WHICH nodes (LoRA adapters, KV caches) move between HBM and host memory; the block lists of
+ * the chosen nodes then go to fl_swap_out / fl_swap_in.  A node is described by what the usage
+ * dependency tree records for it (Section 4.3): kind, where it lives, size, visit count, last use. */
+enum { FL_NODE_LORA = 0, FL_NODE_KV = 1 };
+typedef struct {
+  int32_t kind;         /* FL_NODE_LORA or FL_NODE_KV */
+  int32_t in_hbm;       /* non-zero: resident in HBM; zero: in host memory */
+  int32_t candidate;    /* non-zero: the tree offers this node (an HBM leaf for swap-out, the root of a
+                           host-resident path for swap-in, Section 4.2) */
+  uint32_t n_blocks;    /* size in pool blocks */
+  double visits;        /* visit count of the node */
+  double last_use_s;    /* time of its last use, seconds */
+} fl_node_stat;
+typedef struct {
+  double now_s;             /* current time, seconds (t_i = now_s - last_use_s) */
+  double total_visits;      /* prob_i = visits_i / total_visits */
+  double low_lora;          /* Eq. 3, see fl_expected_lora_demand */
+  int32_t now_lora;         /* adapters resident in HBM now */
+  size_t block_bytes;
+  double link_bytes_per_s;  /* host link bandwidth: cost_i = node bytes / bandwidth (Section 5.2) */
+  double upper, lower;      /* HBM usage thresholds of the monitor tick (the paper uses 0.95 and 0.70) */
+} fl_swap_params;
+/* Eq. 3: expected number of distinct adapters a batch of `batch_size` queries needs,
+ * sum_i (1 - (1 - prob_i)^batch_size).  prob: host pointer, n values in [0, 1]. */
+int fl_expected_lora_demand(const double* prob, int n, int batch_size, double* low_lora);
+/* Eq. 4 - Eq. 6 for every node: eval[i] = LoRA_Eval_i * cost_i * prob_i * (1 - sigmoid(t_i)), with
+ * LoRA_Eval_i = max(1, low_lora / now_lora) for LoRA nodes and 1 for KV nodes (the coefficient rewards
+ * loading adapters while fewer are resident than the batch is expected to need).  A higher value means
+ * more benefit from keeping the node in HBM.  eval: host pointer, n doubles. */
+int fl_swap_eval(const fl_node_stat* nodes, int n, const fl_swap_params* prm, double* eval);
+/* One monitor tick (Section 5.3).  usage = blocks_used / blocks_total.  usage > upper: swap-out, candidates
+ * resident in HBM in ascending eval, one by one until usage <= upper (*direction = -1).  usage < lower:
+ * swap-in, candidates in host memory in descending eval, one by one until usage >= lower, skipping a node
+ * that would push usage above upper (*direction = +1).  Otherwise nothing (*direction = 0, *n_order = 0).
+ * Equal evals keep the lower node index first.  order: host pointer with room for n indices. */
+int fl_swapper_decide(const fl_node_stat* nodes, int n, const fl_swap_params* prm, uint32_t blocks_used,
+                      uint32_t blocks_total, int32_t* order, int* n_order, int* direction);
+
 #ifdef __cplusplus
 }
 #endif

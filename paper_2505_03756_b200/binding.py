@@ -33,6 +33,16 @@ class fl_lora_shape(C.Structure):
     _fields_ = [("d_in", C.c_int32), ("d_out", C.c_int32)]
 
 
+class fl_node_stat(C.Structure):
+    _fields_ = [("kind", C.c_int32), ("in_hbm", C.c_int32), ("candidate", C.c_int32), ("n_blocks", C.c_uint32),
+                ("visits", C.c_double), ("last_use_s", C.c_double)]
+
+
+class fl_swap_params(C.Structure):
+    _fields_ = [("now_s", C.c_double), ("total_visits", C.c_double), ("low_lora", C.c_double), ("now_lora", C.c_int32),
+                ("block_bytes", C.c_size_t), ("link_bytes_per_s", C.c_double), ("upper", C.c_double), ("lower", C.c_double)]
+
+
 class fl_status(C.Structure):
     _fields_ = [("device_flags", C.c_uint32), ("blocks_used", C.c_uint32), ("blocks_free", C.c_uint32),
                 ("host_blocks_used", C.c_uint32), ("host_blocks_free", C.c_uint32), ("lora_blocks", C.c_uint32),
@@ -73,6 +83,10 @@ _SIGS = {
     "fl_swap_in": (C.c_int, [_vp, _vp, _vp, C.c_uint32, _vp]),
     "fl_swap_record": (C.c_int, [_vp, _vp, _vp]),
     "fl_swap_wait": (C.c_int, [_vp, _vp, C.c_int]),
+    "fl_expected_lora_demand": (C.c_int, [_vp, C.c_int, C.c_int, C.POINTER(C.c_double)]),
+    "fl_swap_eval": (C.c_int, [C.POINTER(fl_node_stat), C.c_int, C.POINTER(fl_swap_params), _vp]),
+    "fl_swapper_decide": (C.c_int, [C.POINTER(fl_node_stat), C.c_int, C.POINTER(fl_swap_params), C.c_uint32, C.c_uint32,
+                                    _vp, C.POINTER(C.c_int), C.POINTER(C.c_int)]),
 }
 for _n, (_r, _a) in _SIGS.items():
     getattr(lib, _n).restype = _r
@@ -285,6 +299,49 @@ def fl_swap_record(pool, event, side_stream):
 
 def fl_swap_wait(pool, event, timeout_ms):
     return lib.fl_swap_wait(pool, event.cuda_event, timeout_ms)
+
+
+# ------------------------------------------------------------------ cache swapper (host side)
+FL_NODE_LORA, FL_NODE_KV = 0, 1
+
+
+def _nodes(nodes):
+    arr = (fl_node_stat * len(nodes))()
+    for k, nd in enumerate(nodes):
+        arr[k].kind, arr[k].in_hbm, arr[k].candidate = int(nd["kind"]), int(nd["in_hbm"]), int(nd["candidate"])
+        arr[k].n_blocks, arr[k].visits, arr[k].last_use_s = int(nd["n_blocks"]), float(nd["visits"]), float(nd["last_use_s"])
+    return arr
+
+
+def _params(prm):
+    p = fl_swap_params()
+    for name, _ in fl_swap_params._fields_:
+        setattr(p, name, prm[name])
+    return p
+
+
+def fl_expected_lora_demand(prob, batch_size):
+    prob = np.ascontiguousarray(prob, dtype=np.float64)
+    out = C.c_double()
+    _check(lib.fl_expected_lora_demand(prob.ctypes.data, len(prob), batch_size, C.byref(out)), "fl_expected_lora_demand")
+    return out.value
+
+
+def fl_swap_eval(nodes, prm):
+    arr = nodes if isinstance(nodes, C.Array) else _nodes(nodes)
+    out = np.empty(len(arr), dtype=np.float64)
+    _check(lib.fl_swap_eval(arr, len(arr), C.byref(_params(prm)), out.ctypes.data), "fl_swap_eval")
+    return out
+
+
+def fl_swapper_decide(nodes, prm, blocks_used, blocks_total):
+    """Returns (direction, ordered node indices): -1 swap-out, +1 swap-in, 0 nothing."""
+    arr = nodes if isinstance(nodes, C.Array) else _nodes(nodes)
+    order = np.empty(len(arr), dtype=np.int32)
+    n, d = C.c_int(), C.c_int()
+    _check(lib.fl_swapper_decide(arr, len(arr), C.byref(_params(prm)), blocks_used, blocks_total, order.ctypes.data,
+                                 C.byref(n), C.byref(d)), "fl_swapper_decide")
+    return d.value, order[:n.value].tolist()
 
 
 # ------------------------------------------------------------------ views of the two slabs (for tests and tools)

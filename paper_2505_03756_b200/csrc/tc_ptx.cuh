@@ -109,25 +109,6 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
   return d;
 }
 
-// 2^x for a pair of arguments x <= 126 on the FMA and integer pipes (no special-function unit):
-// x is clamped at -126, split into a rounded integer n and f in [-0.5, 0.5], 2^f comes from a cubic
-// fitted on that interval (relative error 7.5e-5, far below one bf16 rounding), and n is added to the
-// exponent field.  -inf gives 2^-126.
-__device__ __forceinline__ float2 ex2_poly2(float2 x) {
-  const float2 magic = make_float2(12582912.f, 12582912.f);    // 1.5 * 2^23
-  x.x = fmaxf(x.x, -126.f);
-  x.y = fmaxf(x.y, -126.f);
-  const float2 t = __fadd2_rn(x, magic);                        // n sits in the low mantissa bits
-  const float2 n = __fadd2_rn(t, make_float2(-12582912.f, -12582912.f));
-  const float2 f = __ffma2_rn(n, make_float2(-1.f, -1.f), x);
-  float2 p = __ffma2_rn(make_float2(0.0551716648f, 0.0551716648f), f, make_float2(0.2426111400f, 0.2426111400f));
-  p = __ffma2_rn(p, f, make_float2(0.6932609677f, 0.6932609677f));
-  p = __ffma2_rn(p, f, make_float2(0.9999280572f, 0.9999280572f));
-  p.x = __int_as_float(__float_as_int(p.x) + (__float_as_int(t.x) << 23));
-  p.y = __int_as_float(__float_as_int(p.y) + (__float_as_int(t.y) << 23));
-  return p;
-}
-
 // Shared-memory matrix descriptor, 128-byte swizzle (layout code 2), descriptor version 1.
 // K-major operands: lbo unused (1), sbo = 1024 (8 rows of 128 bytes).  MN-major: lbo = distance
 // between 64-element groups along MN, sbo = 1024 (8 rows along K).

@@ -111,6 +111,11 @@ class ClockSampler(threading.Thread):
 
     def result(self):
         self.stop_flag = True
+        if self.nv is not None and not self.samples:      # a timed region shorter than one sampling period
+            try:
+                self.samples.append(self.nv.nvmlDeviceGetClockInfo(self.h, self.nv.NVML_CLOCK_SM))
+            except Exception:
+                pass
         if self.nv is None or not self.samples:
             return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "note": "NVML unavailable"}
         return {"sm_mhz": float(np.median(self.samples)), "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
@@ -385,14 +390,15 @@ def run_ours(args, wl):
                 main.wait_event(ev_side)
                 main.wait_event(ev_side_in)
             nbytes = n_swap * s.block_bytes
-            hp = torch.empty(2 * nbytes, dtype=torch.uint8).pin_memory()
-            dp = torch.empty(2 * nbytes, dtype=torch.uint8, device=dev)
+            lbytes = max(nbytes, 256 << 20)       # the link's peak is taken on copies large enough to reach it
+            hp = torch.empty(2 * lbytes, dtype=torch.uint8).pin_memory()
+            dp = torch.empty(2 * lbytes, dtype=torch.uint8, device=dev)
 
             def link_once():
                 with torch.cuda.stream(side):
-                    hp[:nbytes].copy_(dp[:nbytes], non_blocking=True)
+                    hp[:lbytes].copy_(dp[:lbytes], non_blocking=True)
                 with torch.cuda.stream(side_in):
-                    dp[nbytes:].copy_(hp[nbytes:], non_blocking=True)
+                    dp[lbytes:].copy_(hp[lbytes:], non_blocking=True)
                 ev_side.record(side)
                 ev_side_in.record(side_in)
                 main.wait_event(ev_side)
@@ -408,11 +414,11 @@ def run_ours(args, wl):
                 g1.record(main)
                 barrier()
                 res[name] = g0.elapsed_time(g1) / 5
+            gbs, peak = nbytes / res["swap"] / 1e6, lbytes / res["link"] / 1e6
             swap = {"ms": round(res["swap"], 4), "bytes_each_way": nbytes, "bound": "host link",
-                    "gbs_each_way": round(nbytes / res["swap"] / 1e6, 2),
-                    "link_peak_gbs_each_way": round(nbytes / res["link"] / 1e6, 2),
-                    "frac_link": round(res["link"] / res["swap"], 4),
-                    "note": "both directions at once; peak = two contiguous pinned copies of the same size, measured here"}
+                    "gbs_each_way": round(gbs, 2), "link_peak_gbs_each_way": round(peak, 2), "frac_link": round(gbs / peak, 4),
+                    "note": "both directions at once; peak = two contiguous pinned copies of %d MiB each, one per direction, "
+                            "at once, measured here" % (lbytes >> 20)}
     flags = sess.status()["device_flags"]
     (ms_total, ms_e2e), tokens_all = reduce_over_ranks([ms_total, ms_e2e], T, world, dev)
     ms_step = ms_total / args.steps

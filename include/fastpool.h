@@ -257,6 +257,45 @@ int fl_swap_eval(const fl_node_stat* nodes, int n, const fl_swap_params* prm, do
 int fl_swapper_decide(const fl_node_stat* nodes, int n, const fl_swap_params* prm, uint32_t blocks_used,
                       uint32_t blocks_total, int32_t* order, int* n_order, int* direction);
 
+/* ---------------------------------------------------------------- usage dependency tree (Section 4; host code)
+ * Virtual root -> LoRA nodes (second layer) -> KV nodes, one per pool block of block_tokens tokens, labelled
+ * by those tokens; conversations with a common prefix share its nodes.  The tree only records block ids
+ * ("without altering the physical allocation", Section 4.3); the caller allocates, frees and swaps blocks.
+ * Node ids are dense, starting at 0, in creation order; fl_tree_stats index i describes node i, so the order
+ * fl_swapper_decide returns is a list of node ids. */
+typedef struct fl_tree fl_tree;
+int fl_tree_create(fl_tree** out, int block_tokens);
+int fl_tree_destroy(fl_tree* tree);
+/* Adds the node of adapter lora_id with its block table (device blocks if in_hbm, else host blocks).
+ * FL_EBADID if the adapter has a node already.  *node (may be NULL) receives the node id. */
+int fl_tree_add_lora(fl_tree* tree, int32_t lora_id, const uint32_t* blocks, uint32_t n_blocks, int in_hbm,
+                     double now_s, int32_t* node);
+/* Matching of an arriving query (Section 4.2): its LoRA node, then KV nodes depth first, one per whole block
+ * of `tokens`, until no child carries the next block_tokens tokens.  kv_nodes[0..*n_kv_nodes) is the matched
+ * path (cap entries available, FL_ENOMEM if too few), *matched_tokens = *n_kv_nodes * block_tokens.  Every
+ * matched node (the LoRA node included) gets one visit and last use = now_s.  Nodes that live in host memory
+ * are still matched: the caller swaps them in (root first) before the query runs.  FL_EBADID: unknown adapter. */
+int fl_tree_match(fl_tree* tree, int32_t lora_id, const int32_t* tokens, int n_tokens, double now_s,
+                  int32_t* lora_node, int32_t* kv_nodes, int cap, int* n_kv_nodes, int* matched_tokens);
+/* Inserts n_new_blocks KV nodes as a chain below `parent` (the last matched node, or the LoRA node): node k is
+ * labelled tokens[k * block_tokens ..) and records device block block_ids[k].  New KV is generated in HBM, so
+ * the parent must be in HBM (FL_EBUSY).  FL_EBADID if such a child exists already.  new_nodes may be NULL. */
+int fl_tree_insert(fl_tree* tree, int32_t parent, const int32_t* tokens, int n_new_blocks, const uint32_t* block_ids,
+                   double now_s, int32_t* new_nodes);
+int fl_tree_size(fl_tree* tree);
+int fl_tree_node_blocks(fl_tree* tree, int32_t node, uint32_t* blocks, uint32_t cap, uint32_t* n_blocks);
+/* What the cache swapper needs (Section 5.3): one fl_node_stat per node, with `candidate` set for HBM nodes
+ * without a child in HBM (the only nodes that may be swapped out) and for host nodes whose parent is in HBM or
+ * is the virtual root (the only nodes that may be swapped in); the visit total (prob_i = visits_i / total) and
+ * the number of adapters in HBM.  out may be NULL to query *n_nodes only. */
+int fl_tree_stats(fl_tree* tree, fl_node_stat* out, int cap, int* n_nodes, double* total_visits, int32_t* now_lora);
+/* Records a finished swap of `node` with its new block ids.  FL_EBUSY if the move would break the rule of
+ * Section 4.2 (a node with a child in HBM may not leave; a node whose parent is in host memory may not enter). */
+int fl_tree_set_location(fl_tree* tree, int32_t node, int in_hbm, const uint32_t* blocks, uint32_t n_blocks);
+/* Verifies that every node in HBM has its parent in HBM ("all KV caches that reside in the HBM are valid").
+ * FL_EBADID and *first_bad (may be NULL) on a violation. */
+int fl_tree_check(fl_tree* tree, int32_t* first_bad);
+
 #ifdef __cplusplus
 }
 #endif

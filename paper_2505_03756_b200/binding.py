@@ -83,6 +83,17 @@ _SIGS = {
     "fl_swap_in": (C.c_int, [_vp, _vp, _vp, C.c_uint32, _vp]),
     "fl_swap_record": (C.c_int, [_vp, _vp, _vp]),
     "fl_swap_wait": (C.c_int, [_vp, _vp, C.c_int]),
+    "fl_tree_create": (C.c_int, [C.POINTER(_vp), C.c_int]),
+    "fl_tree_destroy": (C.c_int, [_vp]),
+    "fl_tree_add_lora": (C.c_int, [_vp, C.c_int32, _vp, C.c_uint32, C.c_int, C.c_double, _i32p]),
+    "fl_tree_match": (C.c_int, [_vp, C.c_int32, _vp, C.c_int, C.c_double, _i32p, _vp, C.c_int, C.POINTER(C.c_int),
+                                C.POINTER(C.c_int)]),
+    "fl_tree_insert": (C.c_int, [_vp, C.c_int32, _vp, C.c_int, _vp, C.c_double, _vp]),
+    "fl_tree_size": (C.c_int, [_vp]),
+    "fl_tree_node_blocks": (C.c_int, [_vp, C.c_int32, _vp, C.c_uint32, _u32p]),
+    "fl_tree_stats": (C.c_int, [_vp, C.POINTER(fl_node_stat), C.c_int, C.POINTER(C.c_int), C.POINTER(C.c_double), _i32p]),
+    "fl_tree_set_location": (C.c_int, [_vp, C.c_int32, C.c_int, _vp, C.c_uint32]),
+    "fl_tree_check": (C.c_int, [_vp, _i32p]),
     "fl_expected_lora_demand": (C.c_int, [_vp, C.c_int, C.c_int, C.POINTER(C.c_double)]),
     "fl_swap_eval": (C.c_int, [C.POINTER(fl_node_stat), C.c_int, C.POINTER(fl_swap_params), _vp]),
     "fl_swapper_decide": (C.c_int, [C.POINTER(fl_node_stat), C.c_int, C.POINTER(fl_swap_params), C.c_uint32, C.c_uint32,
@@ -342,6 +353,78 @@ def fl_swapper_decide(nodes, prm, blocks_used, blocks_total):
     _check(lib.fl_swapper_decide(arr, len(arr), C.byref(_params(prm)), blocks_used, blocks_total, order.ctypes.data,
                                  C.byref(n), C.byref(d)), "fl_swapper_decide")
     return d.value, order[:n.value].tolist()
+
+
+# ------------------------------------------------------------------ usage dependency tree (host side)
+def fl_tree_create(block_tokens):
+    h = _vp()
+    _check(lib.fl_tree_create(C.byref(h), block_tokens), "fl_tree_create")
+    return h
+
+
+def fl_tree_destroy(tree):
+    _check(lib.fl_tree_destroy(tree), "fl_tree_destroy")
+
+
+def fl_tree_add_lora(tree, lora_id, blocks, in_hbm, now_s):
+    ids, p = _ids(blocks)
+    node = C.c_int32()
+    _check(lib.fl_tree_add_lora(tree, lora_id, p, len(ids), int(in_hbm), now_s, C.byref(node)), "fl_tree_add_lora")
+    return node.value
+
+
+def fl_tree_match(tree, lora_id, tokens, now_s):
+    """Returns (LoRA node, [matched KV nodes in path order], matched token count)."""
+    tok = np.ascontiguousarray(tokens, dtype=np.int32)
+    cap = len(tok) + 1
+    path = np.empty(cap, dtype=np.int32)
+    ln, n, m = C.c_int32(), C.c_int(), C.c_int()
+    _check(lib.fl_tree_match(tree, lora_id, tok.ctypes.data, len(tok), now_s, C.byref(ln), path.ctypes.data, cap,
+                             C.byref(n), C.byref(m)), "fl_tree_match")
+    return ln.value, path[:n.value].tolist(), m.value
+
+
+def fl_tree_insert(tree, parent, tokens, block_ids, now_s):
+    tok = np.ascontiguousarray(tokens, dtype=np.int32)
+    ids, p = _ids(block_ids)
+    new = np.empty(len(ids), dtype=np.int32)
+    _check(lib.fl_tree_insert(tree, parent, tok.ctypes.data, len(ids), p, now_s, new.ctypes.data), "fl_tree_insert")
+    return new.tolist()
+
+
+def fl_tree_size(tree):
+    return lib.fl_tree_size(tree)
+
+
+def fl_tree_node_blocks(tree, node):
+    n = C.c_uint32()
+    _check(lib.fl_tree_node_blocks(tree, node, None, 0, C.byref(n)), "fl_tree_node_blocks")
+    out = np.empty(n.value, dtype=np.uint32)
+    _check(lib.fl_tree_node_blocks(tree, node, out.ctypes.data, n.value, C.byref(n)), "fl_tree_node_blocks")
+    return out.tolist()
+
+
+def fl_tree_stats(tree, raw=False):
+    """Returns (per-node stats, total visits, adapters in HBM); raw=True keeps the ctypes array for fl_swapper_decide."""
+    n = C.c_int()
+    _check(lib.fl_tree_stats(tree, None, 0, C.byref(n), None, None), "fl_tree_stats")
+    arr = (fl_node_stat * max(1, n.value))()
+    tot, nl = C.c_double(), C.c_int32()
+    _check(lib.fl_tree_stats(tree, arr, n.value, C.byref(n), C.byref(tot), C.byref(nl)), "fl_tree_stats")
+    if raw:
+        return arr, n.value, tot.value, nl.value
+    stats = [{k: getattr(arr[i], k) for k, _ in fl_node_stat._fields_} for i in range(n.value)]
+    return stats, tot.value, nl.value
+
+
+def fl_tree_set_location(tree, node, in_hbm, blocks):
+    ids, p = _ids(blocks)
+    _check(lib.fl_tree_set_location(tree, node, int(in_hbm), p, len(ids)), "fl_tree_set_location")
+
+
+def fl_tree_check(tree):
+    bad = C.c_int32(-1)
+    return lib.fl_tree_check(tree, C.byref(bad)), bad.value
 
 
 # ------------------------------------------------------------------ views of the two slabs (for tests and tools)

@@ -264,14 +264,9 @@ def run_ours(args, wl):
     # shrink + expand per SGMV call, KV append, plan + prefill + decode + merge, swap gather + scatter
     launches_per_step = 2 + 1 + 4 + 2 + (4 if s.inter else 0) + (2 * -(-n_swap // 256) if n_swap > 1 else 0)
 
-    def step(k, evs=None, swap=True):
+    def compute(k, evs=None):
+        """The kernels of one step, in order, on the compute stream."""
         sign = wl.scale if k % 2 == 0 else -wl.scale     # y += s*delta, then y -= s*delta: values stay bounded
-        ids = fl.fl_block_alloc(sess.pool, spare)        # a1: the allocator runs every step
-        fl.fl_block_free(sess.pool, ids[::-1])
-        swap = swap and n_swap > 0
-        if swap:                                          # a7: side streams, overlapped
-            fl.fl_swap_out(sess.pool, swap_dev_out, swap_host_out, side)
-            fl.fl_swap_in(sess.pool, swap_dev_in, swap_host_in, side_in)
         mark = (lambda: None) if evs is None else (lambda: evs.append(_rec(torch, main)))
         mark()
         sess.sgmv([d_y["q"], d_y["k"], d_y["v"]], d_x, ["q", "k", "v"], scale=sign, stream=main)
@@ -287,6 +282,20 @@ def run_ours(args, wl):
             mark()
             sess.sgmv([d_y["down"]], d_y["up"], ["down"], scale=sign, stream=main)
             mark()
+
+    graphs = []          # the step's kernels captured once per sign; replayed when graph launches are on
+
+    def step(k, evs=None, swap=True, use_graph=False):
+        ids = fl.fl_block_alloc(sess.pool, spare)        # a1: the allocator runs every step
+        fl.fl_block_free(sess.pool, ids[::-1])
+        swap = swap and n_swap > 0
+        if swap:                                          # a7: side streams, overlapped
+            fl.fl_swap_out(sess.pool, swap_dev_out, swap_host_out, side)
+            fl.fl_swap_in(sess.pool, swap_dev_in, swap_host_in, side_in)
+        if use_graph and graphs:
+            graphs[k % 2].replay()
+        else:
+            compute(k, evs)
         if swap:
             ev_side.record(side)
             ev_side_in.record(side_in)
@@ -303,18 +312,38 @@ def run_ours(args, wl):
         for k in range(args.warmup):
             step(k)
         barrier()
+        launch_mode = "eager"
+        if not args.no_graph:
+            # the step's kernel launches go into two CUDA graphs (one per sign): a step then costs one graph
+            # launch on the host instead of one call into the library per kernel group
+            try:
+                for parity in range(2):
+                    g = torch.cuda.CUDAGraph()
+                    with torch.cuda.graph(g, stream=main):
+                        compute(parity)
+                    graphs.append(g)
+                for k in range(2):
+                    step(k, use_graph=True)
+                barrier()
+                launch_mode = "cuda_graph"
+            except Exception as exc:      # capture refused: time the eager launches and say so
+                graphs.clear()
+                launch_mode = "eager (graph capture failed: %s)" % type(exc).__name__
         sampler = ClockSampler(local)
         sampler.start()
-        evs = []
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record(main)
         for k in range(args.steps):
-            step(k, evs)
+            step(k, use_graph=True)
         e1.record(main)
         barrier()
         clocks = sampler.result()
         ms_total = e0.elapsed_time(e1)
-        # per-call device time from the events recorded between the calls of the timed steps
+        # per-call device time: the same steps launched eagerly with an event between the calls
+        evs = []
+        for k in range(args.steps):
+            step(k, evs)
+        barrier()
         per = len(calls) + 1
         call_ms = {c: 0.0 for c in calls}
         for k in range(args.steps):
@@ -327,7 +356,7 @@ def run_ours(args, wl):
             d_x.view(torch.int16).copy_(h_x, non_blocking=True)
             for m in names:
                 d_y[m].view(torch.int16).copy_(h_y[m], non_blocking=True)
-            step(0)
+            step(0, use_graph=True)
             h_out.copy_(d_y["down" if s.inter else "o"].view(torch.int16), non_blocking=True)
         e2e_steps = max(3, min(args.steps, 20))
         for k in range(2):
@@ -375,7 +404,7 @@ def run_ours(args, wl):
             h0, h1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             h0.record(main)
             for k in range(args.steps):
-                step(k, swap=False)
+                step(k, swap=False, use_graph=True)
             h1.record(main)
             barrier()
             overlap = {"ms_per_step_without_swap": h0.elapsed_time(h1) / args.steps}
@@ -467,7 +496,7 @@ def run_ours(args, wl):
             "roofline": roof, "kernels": kernels, "swap_overlap": overlap, "cpu_baseline": cb,
             "e2e": {"value": tokens_all / (ms_e2e * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": int(h_out.numel() * 2), "ms_per_step": ms_e2e},
-            "gpu_launches": launches_per_step * args.steps, "clocks": clocks, "device_flags": flags,
+            "gpu_launches": launches_per_step * args.steps, "launch_mode": launch_mode, "clocks": clocks, "device_flags": flags,
         }
         print(json.dumps(out))
     sess.close()
@@ -490,6 +519,7 @@ def main():
     ap.add_argument("--workload", default="prefill7b", choices=list(WORKLOAD_TEXT))
     ap.add_argument("--swap-blocks", type=int, default=-1)
     ap.add_argument("--prefill-kernel", type=int, default=-1, help="FL_OPT_PREFILL_KERNEL value (default: the library's)")
+    ap.add_argument("--no-graph", action="store_true", help="launch every step eagerly instead of replaying CUDA graphs")
     ap.add_argument("--n-req", type=int, default=0, help="reduced copy of the workload with this many requests "
                     "(small pool; for profiler captures, not a bench line)")
     args = ap.parse_args()

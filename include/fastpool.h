@@ -14,7 +14,9 @@
  *  - "device pointer" = memory of the pool's GPU, owned by the caller, at least 16-byte aligned;
  *    "host pointer" = ordinary host memory.  The library never frees caller memory.
  *  - bf16 values are passed as raw 16-bit patterns (fl_bf16).  Head dimension is 128.
- *  - Kernel launches are asynchronous on the given stream; a status of FL_OK means "enqueued".
+ *  - Kernel launches are asynchronous on the given stream; a status of FL_OK means "enqueued".  After one
+ *    ordinary call of each kind (which configures its kernels), fl_lora_sgmv, fl_lora_sgmv_multi, fl_kv_append
+ *    and fl_paged_attention only launch kernels on that stream and can be recorded into a CUDA graph.
  *    Kernels never trap: a block id or token position outside the pool makes the thread skip the
  *    access and set a sticky flag that fl_pool_status reports.
  *  - A pool belongs to one device; calls on one pool from several host threads must be serialised

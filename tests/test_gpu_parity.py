@@ -381,3 +381,47 @@ def test_layer_step_tiny(H):
         assert_close(H.dev_to_f32(ty["o"]), ref["o"], "o")
     finally:
         s.close()
+
+
+# ------------------------------------------------------------------ the same step replayed from a CUDA graph
+def test_layer_step_replayed_from_cuda_graph_is_bit_identical(H):
+    wl = synth.make_workload("prefill7b", n_req=5, len_range=(60, 300), n_adapters=4)
+    s = _session(H, wl)
+    try:
+        s.fill_prefix_kv()
+        sh, T = wl.shape, wl.n_tokens
+        tx = H.f32_to_dev(wl.x("q"), s.dev)
+        y0 = {m: H.f32_to_dev(wl.y_base(m), s.dev) for m in "qkvo"}
+        ty = {m: y0[m].clone() for m in "qkvo"}
+        attn = torch.zeros(T, sh.n_q_heads, 128, dtype=torch.bfloat16, device=s.dev)
+        main = torch.cuda.Stream()
+
+        def compute():
+            s.sgmv([ty["q"], ty["k"], ty["v"]], tx, ["q", "k", "v"], stream=main)
+            s.kv_append(ty["k"], ty["v"], stream=main)
+            s.attention(attn, ty["q"], stream=main)
+            s.sgmv([ty["o"]], attn.view(T, -1), ["o"], stream=main)
+
+        with torch.cuda.stream(main):
+            compute()                                   # eager (also the first-use set-up of every kernel)
+            main.synchronize()
+            want = {m: ty[m].clone() for m in "qkvo"}
+            want_attn = attn.clone()
+            g = torch.cuda.CUDAGraph()
+            for m in "qkvo":
+                ty[m].copy_(y0[m])
+            main.synchronize()
+            with torch.cuda.graph(g, stream=main):
+                compute()
+            for _ in range(2):                          # replay twice from the same inputs
+                for m in "qkvo":
+                    ty[m].copy_(y0[m])
+                attn.zero_()
+                g.replay()
+                main.synchronize()
+                for m in "qkvo":
+                    assert torch.equal(ty[m], want[m]), m
+                assert torch.equal(attn, want_attn)
+        assert s.status()["device_flags"] == 0
+    finally:
+        s.close()

@@ -40,7 +40,7 @@ constexpr uint32_t TILE_BYTES = 2 * HALF_BYTES;        // a Q, K or V tile
 constexpr uint32_t OFF_Q2 = 0;                         // Q_A, Q_B
 constexpr uint32_t OFF_RING = 2 * TILE_BYTES;
 constexpr uint32_t OFF_BAR2 = OFF_RING + NSLOT * TILE_BYTES;
-constexpr uint32_t T2_SMEM = OFF_BAR2 + 256;
+constexpr uint32_t T2_SMEM = OFF_BAR2 + 512;           // barriers, TMEM address, abort flag, two unit descriptors
 constexpr uint32_t T2_TMEM_COLS = 512;                 // S_A | S_B | O_A | O_B, 128 columns each
 constexpr float RESCALE_LOG2 = 8.f;
 
@@ -55,10 +55,12 @@ struct Unit {           // what a CTA works on at one time
   int lim0[2];          // last visible key of row 0 of each tile
   int n_kt[2];          // K/V tiles each tile takes part in
   int n_kt_max, n_pages, tbl0, h;
-  bool valid;
+  int valid;            // 0: the unit's table is too short for its keys (skipped by every role)
+  int index;            // -1 = no more work
 };
 
-// Unit u = (plan tile u / heads_per_item, head slot u % heads_per_item).  Every role decodes it by itself.
+// Unit u = (plan tile u / heads_per_item, head slot u % heads_per_item), decoded once by the producer and handed
+// to the other roles through shared memory.
 __device__ __forceinline__ Unit decode_unit(const AttnArgs& a, int u, int heads_per_item) {
   Unit t;
   const int item = u / heads_per_item, hslot = u % heads_per_item;
@@ -86,6 +88,7 @@ __device__ __forceinline__ Unit decode_unit(const AttnArgs& a, int u, int heads_
   t.tbl0 = a.tbl_indptr[i];
   t.n_pages = (kv_end + BT - 1) / BT;
   t.valid = t.rows[0] >= 1 && t.n_pages >= 1 && t.n_pages <= a.tbl_indptr[i + 1] - t.tbl0;
+  t.index = u;
   return t;
 }
 
@@ -105,7 +108,8 @@ attn_prefill_tc2_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap kv
   auto bar = [&](int k) { return bar0 + 8u * k; };
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + OFF_BAR2 + 8 * C_COUNT);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + OFF_BAR2 + 8 * C_COUNT + 4);
-  volatile int* unit_slot = reinterpret_cast<volatile int*>(smem + OFF_BAR2 + 8 * C_COUNT + 8);   // [2]
+  Unit* unit_slot = reinterpret_cast<Unit*>(smem + OFF_BAR2 + 8 * C_COUNT + 8);   // [2]
+  static_assert(8 * C_COUNT + 8 + 2 * sizeof(Unit) <= 512, "barrier area too small");
 
   if (tid == 0) {
     mbar_init(bar(C_QFULL), 1);
@@ -133,12 +137,14 @@ attn_prefill_tc2_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap kv
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
 
-  // Readers take the k-th unit of this CTA from slot k & 1 (-1 = no more work) and release the slot.
-  auto read_unit = [&](int k, bool arrive) -> int {
-    if (!mbar_wait(bar(C_UFULL + (k & 1)), (k >> 1) & 1, abort_flag)) return -1;
-    const int u = unit_slot[k & 1];
+  // Readers take the k-th unit of this CTA from slot k & 1 (index -1 = no more work) and release the slot.
+  auto read_unit = [&](int k, bool arrive) -> Unit {
+    Unit t;
+    t.index = -1;
+    if (!mbar_wait(bar(C_UFULL + (k & 1)), (k >> 1) & 1, abort_flag)) return t;
+    t = unit_slot[k & 1];
     if (arrive) mbar_arrive(bar(C_UEMPTY + (k & 1)));
-    return u;
+    return t;
   };
 
   // the softmax warpgroups keep 128 scores per thread in registers: they take the registers the third
@@ -151,12 +157,13 @@ attn_prefill_tc2_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap kv
       int n_valid = 0;                 // units whose Q tiles were loaded so far
       for (int k = 0;; ++k) {
         if (k >= 2 && !mbar_wait(bar(C_UEMPTY + (k & 1)), ((k >> 1) - 1) & 1, abort_flag)) break;
-        int u = k == 0 ? (int)blockIdx.x : (int)gridDim.x + atomicAdd(&a.hdr->next_unit, 1);
-        if (u >= n_units) u = -1;
-        unit_slot[k & 1] = u;
+        const int u = k == 0 ? (int)blockIdx.x : (int)gridDim.x + atomicAdd(&a.hdr->next_unit, 1);
+        Unit t;
+        if (u < n_units) t = decode_unit(a, u, heads_per_item);
+        else t.index = -1;
+        unit_slot[k & 1] = t;
         mbar_arrive(bar(C_UFULL + (k & 1)));
-        if (u < 0) break;
-        const Unit t = decode_unit(a, u, heads_per_item);
+        if (t.index < 0) break;
         if (!t.valid) {
           atomicOr(a.pv.flags, (uint32_t)FLAG_BAD_POS);
           continue;
@@ -234,9 +241,8 @@ attn_prefill_tc2_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap kv
       };
       bool ok = true;
       for (int k = 0; ok; ++k) {
-        const int u = read_unit(k, true);
-        if (u < 0) break;
-        const Unit t = decode_unit(a, u, heads_per_item);
+        const Unit t = read_unit(k, true);
+        if (t.index < 0) break;
         if (!t.valid) continue;
         const int n_kt = t.n_kt_max, nA = t.n_kt[0], nB = t.n_kt[1];
         const int base = cons;         // ring index of K_0 of this unit; K_j = base + 2j, V_j = base + 2j + 1
@@ -284,15 +290,16 @@ attn_prefill_tc2_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap kv
     int steps = 0;      // S tiles of this tile taken so far (phase of C_SFULL)
     int epis = 0;       // epilogues so far (phase of C_ODONE)
     for (int k = 0;; ++k) {
-      const int u = read_unit(k, false);
+      // this tile's few fields straight from the published descriptor
+      if (!mbar_wait(bar(C_UFULL + (k & 1)), (k >> 1) & 1, abort_flag)) break;
+      const Unit* up = unit_slot + (k & 1);
+      const int u_index = up->index, u_valid = up->valid;
+      const int rows = up->rows[x], nk = up->n_kt[x], lim0 = up->lim0[x], out_tok0 = up->tok0[x], out_hq = up->hq[x];
       __syncwarp();
-      if (lane == 0 && u >= 0) mbar_arrive(bar(C_UEMPTY + (k & 1)));
-      if (u < 0) break;
-      const Unit t = decode_unit(a, u, heads_per_item);
-      if (!t.valid) continue;
-      const int rows = x ? t.rows[1] : t.rows[0], nk = x ? t.n_kt[1] : t.n_kt[0];
-      if (nk == 0) continue;
-      const int lim = row < rows ? (x ? t.lim0[1] : t.lim0[0]) + row : -1;
+      if (lane == 0 && u_index >= 0) mbar_arrive(bar(C_UEMPTY + (k & 1)));
+      if (u_index < 0) break;
+      if (!u_valid || nk == 0) continue;
+      const int lim = row < rows ? lim0 + row : -1;
       float m_used = 0.f, m_run = -INFINITY, l = 0.f;
       bool ok = true;
       for (int j = 0; j < nk; ++j) {
@@ -367,7 +374,7 @@ attn_prefill_tc2_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap kv
       if (!ok) break;
       tc_fence_after();
       const float inv = l > 0.f ? 1.f / l : 0.f;
-      uint4* orow = reinterpret_cast<uint4*>(a.out + ((size_t)((x ? t.tok0[1] : t.tok0[0]) + row) * a.n_q + (x ? t.hq[1] : t.hq[0])) * D);
+      uint4* orow = reinterpret_cast<uint4*>(a.out + ((size_t)(out_tok0 + row) * a.n_q + out_hq) * D);
 #pragma unroll
       for (int cb = 0; cb < D; cb += 32) {
         uint32_t o[32];

@@ -203,6 +203,128 @@ __global__ void __launch_bounds__(SG_THREADS) sgmv_shrink_kernel(const SgmvArgs 
   }
 }
 
+// The shrink of three projections that share x (q, k, v) for long segments and ranks up to 16: one CTA stages each x tile once and
+// multiplies it by the three adapters' rank-rows, instead of three CTAs reading the same x rows.  With long
+// segments the shrink is bound by the traffic from L2 into shared memory, and x is most of it.
+template <int RMAX>
+__global__ void __launch_bounds__(SG_THREADS) sgmv_shrink3_kernel(const SgmvArgs a) {
+  constexpr int TM = 64, NM = 3;
+  constexpr int STAGES = RMAX == 64 ? 3 : 4;
+  extern __shared__ __align__(128) unsigned char smem[];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int tile = blockIdx.x, split = blockIdx.y;
+  int seg, tok0, tok1;
+  if (!find_tile<TM>(a.seg_indptr, a.lora_ids, a.n_seg, tile, seg, tok0, tok1)) return;
+  const int lid = a.lora_ids[seg];
+  if ((uint32_t)lid >= a.pv.dir_cap || a.pv.dir[lid].rank <= 0) {
+    if (tid == 0) atomicOr(a.pv.flags, (uint32_t)FLAG_BAD_LORA);
+    return;
+  }
+  const LoraEntry* e = a.pv.dir + lid;
+  for (int m = 0; m < NM; ++m) {
+    if (a.mat_index[m] >= e->n_mats) {
+      if (tid == 0) atomicOr(a.pv.flags, (uint32_t)FLAG_BAD_LORA);
+      return;
+    }
+  }
+  const int rank = min(e->rank, RMAX);
+  const uint32_t table_off = e->table_off;
+  const int d_in = e->mats[a.mat_index[0]].d_in;
+  const int kchunk = ((d_in + a.ksplit * KS - 1) / (a.ksplit * KS)) * KS;
+  const int kb = split * kchunk, ke = min(d_in, kb + kchunk);
+  const int n_it = ke > kb ? (ke - kb + KS - 1) / KS : 0;
+
+  constexpr int XR = TM / 16, AR = RMAX / 16;
+  constexpr int STAGE_BYTES = (TM + NM * RMAX) * 128;
+  const int crow = tid >> 3, cchunk = tid & 7;
+  const __nv_bfloat16* xrow[XR];
+  bool xok[XR];
+#pragma unroll
+  for (int i = 0; i < XR; ++i) {
+    const int t = tok0 + crow + 16 * i;
+    xok[i] = t < tok1;
+    xrow[i] = a.x + (size_t)(xok[i] ? t : tok0) * d_in;
+  }
+  const __nv_bfloat16* arow[NM][AR];
+  bool aok[NM][AR];
+#pragma unroll
+  for (int m = 0; m < NM; ++m) {
+    const LoraMat lm = e->mats[a.mat_index[m]];
+#pragma unroll
+    for (int i = 0; i < AR; ++i) {
+      const int r = crow + 16 * i;
+      aok[m][i] = false;
+      arow[m][i] = reinterpret_cast<const __nv_bfloat16*>(a.pv.slab);
+      if (r < rank)
+        arow[m][i] = reinterpret_cast<const __nv_bfloat16*>(
+            lora_row(a.pv, table_off, lm.a_tab, lm.a_row0, lm.a_rpb, d_in, r, aok[m][i]));
+    }
+  }
+  const uint32_t sbase = smem_u32(smem);
+  auto load_stage = [&](int it, int st) {
+    const int kk = kb + it * KS + cchunk * 8;
+    const bool kok = kk < ke;
+    const uint32_t xs = sbase + st * STAGE_BYTES;
+#pragma unroll
+    for (int i = 0; i < XR; ++i) cp_async16(xs + swz(crow + 16 * i, cchunk, 8), xrow[i] + kk, xok[i] && kok);
+#pragma unroll
+    for (int m = 0; m < NM; ++m) {
+      const uint32_t as = xs + (TM + m * RMAX) * 128;
+#pragma unroll
+      for (int i = 0; i < AR; ++i) cp_async16(as + swz(crow + 16 * i, cchunk, 8), arow[m][i] + kk, aok[m][i] && kok);
+    }
+  };
+
+  float acc[NM][RMAX / 8][4];
+#pragma unroll
+  for (int m = 0; m < NM; ++m)
+#pragma unroll
+    for (int n = 0; n < RMAX / 8; ++n) acc[m][n][0] = acc[m][n][1] = acc[m][n][2] = acc[m][n][3] = 0.f;
+
+#pragma unroll
+  for (int s = 0; s < STAGES - 1; ++s) {
+    if (s < n_it) load_stage(s, s);
+    cp_async_commit();
+  }
+  const int mrow = warp * 16 + (lane & 7) + 8 * ((lane >> 3) & 1);
+  for (int it = 0; it < n_it; ++it) {
+    cp_async_wait<STAGES - 2>();
+    __syncthreads();
+    if (it + STAGES - 1 < n_it) load_stage(it + STAGES - 1, (it + STAGES - 1) % STAGES);
+    cp_async_commit();
+    const uint32_t xs = sbase + (it % STAGES) * STAGE_BYTES;
+#pragma unroll
+    for (int ks = 0; ks < KS / 16; ++ks) {
+      uint32_t af[4];
+      ldmatrix_x4(af, xs + swz(mrow, 2 * ks + (lane >> 4), 8));
+#pragma unroll
+      for (int m = 0; m < NM; ++m) {
+        const uint32_t as = xs + (TM + m * RMAX) * 128;
+#pragma unroll
+        for (int p = 0; p < RMAX / 16; ++p) {
+          if (16 * p < rank) {
+            uint32_t bf[4];
+            ldmatrix_x4(bf, as + swz(16 * p + (lane & 7) + 8 * (lane >> 4), 2 * ks + ((lane >> 3) & 1), 8));
+            mma_bf16(acc[m][2 * p], af, bf[0], bf[1]);
+            mma_bf16(acc[m][2 * p + 1], af, bf[2], bf[3]);
+          }
+        }
+      }
+    }
+  }
+  const int g = lane >> 2, t4 = lane & 3;
+  const int r0 = tok0 + warp * 16 + g;
+#pragma unroll
+  for (int m = 0; m < NM; ++m) {
+    float* vout = a.v + ((size_t)(m * a.ksplit + split) * a.n_tokens) * RMAX;
+#pragma unroll
+    for (int n = 0; n < RMAX / 8; ++n) {
+      if (r0 < tok1) *reinterpret_cast<float2*>(vout + (size_t)r0 * RMAX + 8 * n + 2 * t4) = make_float2(acc[m][n][0], acc[m][n][1]);
+      if (r0 + 8 < tok1) *reinterpret_cast<float2*>(vout + (size_t)(r0 + 8) * RMAX + 8 * n + 2 * t4) = make_float2(acc[m][n][2], acc[m][n][3]);
+    }
+  }
+}
+
 template <int TM, int RMAX>
 __global__ void __launch_bounds__(SG_THREADS) sgmv_expand_kernel(const SgmvArgs a) {
   extern __shared__ __align__(128) unsigned char smem[];
@@ -361,7 +483,17 @@ int launch_pair(fl_pool* p, const SgmvArgs& a, int tiles, int d_out_max, cudaStr
     FL_CUDA(p, cudaFuncSetAttribute(sgmv_expand_kernel<TM, RMAX>, cudaFuncAttributeMaxDynamicSharedMemorySize, expand_smem));
     configured[p->device & 15] = true;
   }
-  sgmv_shrink_kernel<TM, RMAX><<<dim3(tiles * a.n_mats, a.ksplit), SG_THREADS, shrink_smem, st>>>(a);
+  if (TM == 64 && RMAX == 16 && a.n_mats == 3) {      // at higher ranks the three accumulators cost too many registers
+    static bool configured3[16] = {};
+    const int smem3 = (RMAX == 64 ? 3 : 4) * (64 + 3 * RMAX) * 128;
+    if (!configured3[p->device & 15]) {
+      FL_CUDA(p, cudaFuncSetAttribute(sgmv_shrink3_kernel<RMAX>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem3));
+      configured3[p->device & 15] = true;
+    }
+    sgmv_shrink3_kernel<RMAX><<<dim3(tiles, a.ksplit), SG_THREADS, smem3, st>>>(a);
+  } else {
+    sgmv_shrink_kernel<TM, RMAX><<<dim3(tiles * a.n_mats, a.ksplit), SG_THREADS, shrink_smem, st>>>(a);
+  }
   sgmv_expand_kernel<TM, RMAX><<<dim3(tiles * a.n_mats, (d_out_max + EXPAND_COLS - 1) / EXPAND_COLS), SG_THREADS, expand_smem, st>>>(a);
   FL_CUDA(p, cudaGetLastError());
   return FL_OK;

@@ -4,7 +4,8 @@
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload prefill7b] [--impl ours|reference]
 
 One step = one pass of the whole hot path over one synthetic batch: block alloc/free for the batch's
-new-token blocks, LoRA q/k/v projection (SGMV), KV append, paged attention over [cached prefix ||
+new-token blocks, LoRA q/k/v projection (SGMV) with the new K, V written into their pool blocks (one fused call,
+or projection and KV append as two calls with --separate-append), paged attention over [cached prefix ||
 new tokens], LoRA o projection (plus up/down when the layer has them), and a block swap-out/swap-in
 on a side stream that overlaps the kernels.  Prints one JSON line (rank 0).
 """
@@ -65,6 +66,8 @@ def work_model(wl):
     attn_bytes = 2 * (2 * T * s.n_q_heads * d) + float(np.sum(p + n)) * 2 * s.n_kv_heads * d * 2
     w = {
         "sgmv_qkv": {"bytes": sgmv_bytes(["q", "k", "v"]), "bound": "hbm"},
+        # k, v: base rows read from y, result rows written into pool blocks: the same byte count as updating y in place
+        "sgmv_qkv_append": {"bytes": sgmv_bytes(["q", "k", "v"]), "bound": "hbm"},
         "kv_append": {"bytes": 2 * 2 * T * s.n_kv_heads * d * 2, "bound": "hbm"},
         "attention": {"bytes": attn_bytes, "flops": attn_flops,
                       "bound": "tensor" if attn_flops / attn_bytes > 200 else "hbm"},
@@ -260,18 +263,23 @@ def run_ours(args, wl):
     main = torch.cuda.Stream()
     side, side_in = torch.cuda.Stream(), torch.cuda.Stream()      # swap-out and swap-in overlap each other too
     ev_side, ev_side_in = torch.cuda.Event(), torch.cuda.Event()
-    calls = ["sgmv_qkv", "kv_append", "attention", "sgmv_o"] + (["sgmv_up", "sgmv_down"] if s.inter else [])
+    calls = (["sgmv_qkv", "kv_append"] if args.separate_append else ["sgmv_qkv_append"]) + ["attention", "sgmv_o"] + \
+        (["sgmv_up", "sgmv_down"] if s.inter else [])
     # shrink + expand per SGMV call, KV append, plan + prefill + decode + merge, swap gather + scatter
-    launches_per_step = 2 + 1 + 4 + 2 + (4 if s.inter else 0) + (2 * -(-n_swap // 256) if n_swap > 1 else 0)
+    launches_per_step = 2 + (1 if args.separate_append else 0) + 4 + 2 + (4 if s.inter else 0) + \
+        (2 * -(-n_swap // 256) if n_swap > 1 else 0)
 
     def compute(k, evs=None):
         """The kernels of one step, in order, on the compute stream."""
         sign = wl.scale if k % 2 == 0 else -wl.scale     # y += s*delta, then y -= s*delta: values stay bounded
         mark = (lambda: None) if evs is None else (lambda: evs.append(_rec(torch, main)))
         mark()
-        sess.sgmv([d_y["q"], d_y["k"], d_y["v"]], d_x, ["q", "k", "v"], scale=sign, stream=main)
-        mark()
-        sess.kv_append(d_y["k"], d_y["v"], stream=main)
+        if args.separate_append:
+            sess.sgmv([d_y["q"], d_y["k"], d_y["v"]], d_x, ["q", "k", "v"], scale=sign, stream=main)
+            mark()
+            sess.kv_append(d_y["k"], d_y["v"], stream=main)
+        else:       # a4 inside a3: the k, v projections write their rows straight into the pool blocks
+            sess.sgmv_qkv_append(d_y["q"], d_y["k"], d_y["v"], d_x, scale=sign, stream=main)
         mark()
         sess.attention(d_attn, d_y["q"], stream=main)
         mark()
@@ -375,6 +383,8 @@ def run_ours(args, wl):
             sign = wl.scale if k % 2 == 0 else -wl.scale
             if c == "sgmv_qkv":
                 sess.sgmv([d_y["q"], d_y["k"], d_y["v"]], d_x, ["q", "k", "v"], scale=sign, stream=main)
+            elif c == "sgmv_qkv_append":
+                sess.sgmv_qkv_append(d_y["q"], d_y["k"], d_y["v"], d_x, scale=sign, stream=main)
             elif c == "kv_append":
                 sess.kv_append(d_y["k"], d_y["v"], stream=main)
             elif c == "attention":
@@ -519,6 +529,8 @@ def main():
     ap.add_argument("--workload", default="prefill7b", choices=list(WORKLOAD_TEXT))
     ap.add_argument("--swap-blocks", type=int, default=-1)
     ap.add_argument("--prefill-kernel", type=int, default=-1, help="FL_OPT_PREFILL_KERNEL value (default: the library's)")
+    ap.add_argument("--separate-append", action="store_true", help="q/k/v projection and KV append as two calls "
+                    "(default: one call whose k, v results go straight into the pool blocks)")
     ap.add_argument("--no-graph", action="store_true", help="launch every step eagerly instead of replaying CUDA graphs")
     ap.add_argument("--n-req", type=int, default=0, help="reduced copy of the workload with this many requests "
                     "(small pool; for profiler captures, not a bench line)")

@@ -149,6 +149,21 @@ int fl_lora_sgmv_multi(fl_pool* pool, fl_bf16* const* ys, const fl_bf16* x, cons
                        const int32_t* seg_indptr, const int32_t* lora_ids, int n_seg, int n_tokens,
                        float scale, void* workspace, size_t workspace_bytes, fl_stream stream);
 
+/* The q, k, v projections of a layer with the KV store folded in (Eq. 2 and Section 4.3 in one pass: the K/V a
+ * query generates "is directly retained in the HBM" blocks).  q is updated in place like fl_lora_sgmv.  For k
+ * and v the base projections are READ from y_k, y_v and the results (base + LoRA term) are WRITTEN only into
+ * the requests' pool blocks, at the positions and in the layout fl_kv_append uses (including the cleared V slots
+ * behind a request's last token); y_k and y_v are left as they were.  The result in the pool is bit for bit
+ * what fl_lora_sgmv_multi followed by fl_kv_append gives, without writing k, v out and reading them back.
+ * Segments with lora_ids[s] < 0 get their base k, v copied into the pool.  mat_k and mat_v must have
+ * d_out = n_kv_heads * 128 and the three projections share x; req_indptr .. prefix_lens as in fl_kv_append;
+ * workspace as in fl_lora_sgmv_multi with n_mats = 3. */
+int fl_lora_sgmv_qkv_append(fl_pool* pool, fl_bf16* y_q, const fl_bf16* y_k, const fl_bf16* y_v, const fl_bf16* x,
+                            int mat_q, int mat_k, int mat_v, const int32_t* seg_indptr, const int32_t* lora_ids,
+                            int n_seg, int n_tokens, float scale, const int32_t* req_indptr,
+                            const int32_t* kv_tbl_indptr, const uint32_t* kv_tbl, const int32_t* prefix_lens,
+                            int n_req, int n_kv_heads, void* workspace, size_t workspace_bytes, fl_stream stream);
+
 /* fl_lora_sgmv without a workspace argument, for callers that cannot allocate device memory.  (The
  * paper has no counterpart; this is a convenience of the library.)  A serving engine that follows the
  * paper hands all of its HBM to the block pool at start-up; once it is serving, a cudaMalloc may fail

@@ -75,6 +75,8 @@ _SIGS = {
     "fl_lora_sgmv_static": (C.c_int, [_vp, _vp, _vp, C.c_int, _vp, _vp, C.c_int, C.c_int, C.c_float, _vp]),
     "fl_lora_sgmv_multi": (C.c_int, [_vp, C.POINTER(_vp), _vp, _i32p, C.c_int, _vp, _vp, C.c_int, C.c_int,
                                      C.c_float, _vp, C.c_size_t, _vp]),
+    "fl_lora_sgmv_qkv_append": (C.c_int, [_vp, _vp, _vp, _vp, _vp, C.c_int, C.c_int, C.c_int, _vp, _vp, C.c_int, C.c_int,
+                                          C.c_float, _vp, _vp, _vp, _vp, C.c_int, C.c_int, _vp, C.c_size_t, _vp]),
     "fl_kv_append": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, C.c_int, C.c_int, C.c_int, _vp]),
     "fl_paged_attention_workspace": (C.c_size_t, [C.c_int, C.c_int, C.c_int, C.c_int, C.c_int]),
     "fl_paged_attention": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, C.c_int, C.c_int, C.c_int, C.c_int,
@@ -268,6 +270,15 @@ def fl_lora_sgmv_multi(pool, ys, x, mat_indices, seg_indptr, lora_ids, n_seg, n_
     _check(lib.fl_lora_sgmv_multi(pool, py, _dev(x), mi, len(ys), _dev(seg_indptr), _dev(lora_ids), n_seg, n_tokens,
                                   scale, _dev(workspace), workspace.numel() * workspace.element_size(),
                                   _stream(stream)), "fl_lora_sgmv_multi")
+
+
+def fl_lora_sgmv_qkv_append(pool, y_q, y_k, y_v, x, mat_q, mat_k, mat_v, seg_indptr, lora_ids, n_seg, n_tokens, scale,
+                            req_indptr, kv_tbl_indptr, kv_tbl, prefix_lens, n_req, n_kv_heads, workspace, stream=None):
+    _check(lib.fl_lora_sgmv_qkv_append(pool, _dev(y_q), _dev(y_k), _dev(y_v), _dev(x), mat_q, mat_k, mat_v,
+                                       _dev(seg_indptr), _dev(lora_ids), n_seg, n_tokens, scale, _dev(req_indptr),
+                                       _dev(kv_tbl_indptr), _dev(kv_tbl), _dev(prefix_lens), n_req, n_kv_heads,
+                                       _dev(workspace), workspace.numel() * workspace.element_size(), _stream(stream)),
+           "fl_lora_sgmv_qkv_append")
 
 
 def fl_kv_append(pool, k_new, v_new, req_indptr, kv_tbl_indptr, kv_tbl, prefix_lens, n_req, n_tokens, n_kv_heads,

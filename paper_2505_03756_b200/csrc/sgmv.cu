@@ -32,13 +32,23 @@ struct SgmvArgs {
   float scale;
   float* v;        // [n_mats][ksplit][n_tokens][RMAX]
   int ksplit;
+  int d_out[FL_MAX_MATS];
+  // K / V projections whose result goes straight into the requests' pool blocks instead of back into y
+  // (kv_side[j] = 0: K, 1: V, -1: y updated in place); then segments without an adapter are tiled too
+  int kv_side[FL_MAX_MATS];
+  int all_segments;
+  const int32_t* req_indptr;
+  const int32_t* tbl_indptr;
+  const uint32_t* tbl;
+  const int32_t* prefix_lens;
+  int n_req, n_kv, bt;
 };
 
-// Token tile `tile` (tiles of TM tokens, counted over segments that carry an adapter) -> segment and
+// Token tile `tile` (tiles of TM tokens, counted over segments that carry an adapter, or over all segments) -> segment and
 // token range.  Every warp evaluates it redundantly with a warp scan over 32 segments at a time.
 template <int TM>
 __device__ __forceinline__ bool find_tile(const int32_t* __restrict__ seg_indptr, const int32_t* __restrict__ lora_ids,
-                                          int n_seg, int tile, int& seg, int& tok0, int& tok1) {
+                                          int n_seg, int tile, int& seg, int& tok0, int& tok1, bool all_segments = false) {
   const int lane = threadIdx.x & 31;
   int base = 0;
   for (int s0 = 0; s0 < n_seg; s0 += 32) {
@@ -47,7 +57,7 @@ __device__ __forceinline__ bool find_tile(const int32_t* __restrict__ seg_indptr
     if (s < n_seg) {
       lo = seg_indptr[s];
       hi = seg_indptr[s + 1];
-      if (lora_ids[s] >= 0 && hi > lo) nt = (hi - lo + TM - 1) / TM;
+      if ((all_segments || lora_ids[s] >= 0) && hi > lo) nt = (hi - lo + TM - 1) / TM;
     }
     int incl = nt;
 #pragma unroll
@@ -93,8 +103,9 @@ __global__ void __launch_bounds__(SG_THREADS) sgmv_shrink_kernel(const SgmvArgs 
   const int tile = blockIdx.x / a.n_mats;
   const int split = blockIdx.y;
   int seg, tok0, tok1;
-  if (!find_tile<TM>(a.seg_indptr, a.lora_ids, a.n_seg, tile, seg, tok0, tok1)) return;
+  if (!find_tile<TM>(a.seg_indptr, a.lora_ids, a.n_seg, tile, seg, tok0, tok1, a.all_segments != 0)) return;
   const int lid = a.lora_ids[seg];
+  if (lid < 0) return;
   if ((uint32_t)lid >= a.pv.dir_cap || a.pv.dir[lid].rank <= 0 || a.mat_index[j] >= a.pv.dir[lid].n_mats) {
     if (tid == 0) atomicOr(a.pv.flags, (uint32_t)FLAG_BAD_LORA);
     return;
@@ -214,8 +225,9 @@ __global__ void __launch_bounds__(SG_THREADS) sgmv_shrink3_kernel(const SgmvArgs
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int tile = blockIdx.x, split = blockIdx.y;
   int seg, tok0, tok1;
-  if (!find_tile<TM>(a.seg_indptr, a.lora_ids, a.n_seg, tile, seg, tok0, tok1)) return;
+  if (!find_tile<TM>(a.seg_indptr, a.lora_ids, a.n_seg, tile, seg, tok0, tok1, a.all_segments != 0)) return;
   const int lid = a.lora_ids[seg];
+  if (lid < 0) return;
   if ((uint32_t)lid >= a.pv.dir_cap || a.pv.dir[lid].rank <= 0) {
     if (tid == 0) atomicOr(a.pv.flags, (uint32_t)FLAG_BAD_LORA);
     return;
@@ -325,21 +337,34 @@ __global__ void __launch_bounds__(SG_THREADS) sgmv_shrink3_kernel(const SgmvArgs
   }
 }
 
-template <int TM, int RMAX>
-__global__ void __launch_bounds__(SG_THREADS) sgmv_expand_kernel(const SgmvArgs a) {
+// KV: some projections of the call write their result rows into pool blocks (SgmvArgs::kv_side).
+// CTAs per SM the register budget is sized for (the kernel is bound by memory latency: occupancy matters more
+// than a few spilled values)
+constexpr int expand_min_ctas(int tm, int rmax, bool) { return tm == 16 ? 5 : (rmax == 16 ? 4 : 3); }
+
+template <int TM, int RMAX, bool KV>
+__global__ void __launch_bounds__(SG_THREADS, expand_min_ctas(TM, RMAX, KV)) sgmv_expand_kernel(const SgmvArgs a) {
   extern __shared__ __align__(128) unsigned char smem[];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int j = blockIdx.x % a.n_mats;
   const int tile = blockIdx.x / a.n_mats;
   int seg, tok0, tok1;
-  if (!find_tile<TM>(a.seg_indptr, a.lora_ids, a.n_seg, tile, seg, tok0, tok1)) return;
+  if (!find_tile<TM>(a.seg_indptr, a.lora_ids, a.n_seg, tile, seg, tok0, tok1, a.all_segments != 0)) return;
   const int lid = a.lora_ids[seg];
-  if ((uint32_t)lid >= a.pv.dir_cap || a.pv.dir[lid].rank <= 0 || a.mat_index[j] >= a.pv.dir[lid].n_mats) return;
-  const LoraEntry* e = a.pv.dir + lid;
-  const LoraMat lm = e->mats[a.mat_index[j]];
-  const int rank = min(e->rank, RMAX);
-  const uint32_t table_off = e->table_off;
-  const int d_out = lm.d_out;
+  const int side = KV ? a.kv_side[j] : -1;   // >= 0: the result rows go into the requests' pool blocks
+  int rank = 0;
+  uint32_t table_off = 0;
+  LoraMat lm = {};
+  if (lid >= 0) {
+    if ((uint32_t)lid >= a.pv.dir_cap || a.pv.dir[lid].rank <= 0 || a.mat_index[j] >= a.pv.dir[lid].n_mats) return;
+    const LoraEntry* e = a.pv.dir + lid;
+    lm = e->mats[a.mat_index[j]];
+    rank = min(e->rank, RMAX);
+    table_off = e->table_off;
+  } else if (side < 0) {
+    return;                                // no adapter and y stays where it is: nothing to do
+  }
+  const int d_out = a.d_out[j];
   const int c0 = blockIdx.y * EXPAND_COLS;
   if (c0 >= d_out) return;
   const int c1 = min(d_out, c0 + EXPAND_COLS);
@@ -387,6 +412,42 @@ __global__ void __launch_bounds__(SG_THREADS) sgmv_expand_kernel(const SgmvArgs 
     const int t = tok0 + crow + 8 * i;
     yok[i] = t < tok1;
     yrow[i] = a.y[j] + (size_t)(yok[i] ? t : tok0) * d_out;
+  }
+  // K / V rows: where each of this thread's token rows lives in the pool (block and slot of its position),
+  // and how many slots behind it have to be cleared (V of a request's last token)
+  uint32_t kvloc[KV ? YR : 1];      // block << 5 | slot << 1 | "last token of its request"
+  if (KV && side >= 0) {
+    int r = 0;
+    {
+      int lo = 0, hi = a.n_req;
+      const int t0 = tok0 + crow;
+      while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (a.req_indptr[mid] <= t0) lo = mid; else hi = mid;
+      }
+      r = lo;
+    }
+#pragma unroll
+    for (int i = 0; i < YR; ++i) {
+      kvloc[i] = 0;
+      const int t = tok0 + crow + 8 * i;
+      if (!yok[i]) continue;
+      while (r + 1 < a.n_req && t >= a.req_indptr[r + 1]) ++r;
+      const int pos = a.prefix_lens[r] + (t - a.req_indptr[r]);
+      const int entry = pos / a.bt, slot = pos - entry * a.bt;
+      if (t < a.req_indptr[r] || t >= a.req_indptr[r + 1] || entry >= a.tbl_indptr[r + 1] - a.tbl_indptr[r]) {
+        atomicOr(a.pv.flags, (uint32_t)FLAG_BAD_POS);
+        yok[i] = false;
+        continue;
+      }
+      const uint32_t blk = a.tbl[a.tbl_indptr[r] + entry];
+      if (blk >= a.pv.n_blocks || blk >= (1u << 27)) {
+        atomicOr(a.pv.flags, (uint32_t)FLAG_BAD_BLOCK);
+        yok[i] = false;
+        continue;
+      }
+      kvloc[i] = blk << 5 | (uint32_t)slot << 1 | (t == a.req_indptr[r + 1] - 1 ? 1u : 0u);
+    }
   }
   const __nv_bfloat16* brow[BR];
   bool bok[BR];
@@ -454,10 +515,28 @@ __global__ void __launch_bounds__(SG_THREADS) sgmv_expand_kernel(const SgmvArgs 
     {
       const int col = c0 + sub * NSUB + cchunk * 8;
       if (col < c1) {
+        if (!KV || side < 0) {
 #pragma unroll
-        for (int i = 0; i < YR; ++i)
-          if (yok[i])
-            *reinterpret_cast<uint4*>(yrow[i] + col) = *reinterpret_cast<const uint4*>(ysm + swz(crow + 8 * i, cchunk, 16));
+          for (int i = 0; i < YR; ++i)
+            if (yok[i])
+              *reinterpret_cast<uint4*>(yrow[i] + col) = *reinterpret_cast<const uint4*>(ysm + swz(crow + 8 * i, cchunk, 16));
+        } else if (KV) {
+          // a sub-tile is one KV head: [K|V][head][slot][128] inside the block
+          static_assert(NSUB == FL_HEAD_DIM, "a sub-tile must be one head");
+          const size_t head_off = ((size_t)side * a.n_kv + (c0 + sub * NSUB) / FL_HEAD_DIM) * a.bt * (FL_HEAD_DIM * 2) + cchunk * 16;
+#pragma unroll
+          for (int i = 0; i < YR; ++i) {
+            if (yok[i]) {
+              const uint32_t loc = kvloc[KV ? i : 0];
+              const int slot = (loc >> 1) & 15;
+              unsigned char* dst = a.pv.slab + (size_t)(loc >> 5) * a.pv.block_bytes + head_off + slot * (FL_HEAD_DIM * 2);
+              *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(ysm + swz(crow + 8 * i, cchunk, 16));
+              if (side == 1 && (loc & 1u))     // V of a request's last token: clear the slots behind it
+                for (int z = slot + 1; z < a.bt; ++z)
+                  *reinterpret_cast<uint4*>(dst + (z - slot) * (FL_HEAD_DIM * 2)) = make_uint4(0u, 0u, 0u, 0u);
+            }
+          }
+        }
       }
     }
     __syncthreads();
@@ -480,7 +559,8 @@ int launch_pair(fl_pool* p, const SgmvArgs& a, int tiles, int d_out_max, cudaStr
   const int expand_smem = 2 * (TM + RMAX) * 256;
   if (!configured[p->device & 15]) {
     FL_CUDA(p, cudaFuncSetAttribute(sgmv_shrink_kernel<TM, RMAX>, cudaFuncAttributeMaxDynamicSharedMemorySize, shrink_smem));
-    FL_CUDA(p, cudaFuncSetAttribute(sgmv_expand_kernel<TM, RMAX>, cudaFuncAttributeMaxDynamicSharedMemorySize, expand_smem));
+    FL_CUDA(p, cudaFuncSetAttribute(sgmv_expand_kernel<TM, RMAX, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, expand_smem));
+    FL_CUDA(p, cudaFuncSetAttribute(sgmv_expand_kernel<TM, RMAX, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, expand_smem));
     configured[p->device & 15] = true;
   }
   if (TM == 64 && RMAX == 16 && a.n_mats == 3) {      // at higher ranks the three accumulators cost too many registers
@@ -494,7 +574,9 @@ int launch_pair(fl_pool* p, const SgmvArgs& a, int tiles, int d_out_max, cudaStr
   } else {
     sgmv_shrink_kernel<TM, RMAX><<<dim3(tiles * a.n_mats, a.ksplit), SG_THREADS, shrink_smem, st>>>(a);
   }
-  sgmv_expand_kernel<TM, RMAX><<<dim3(tiles * a.n_mats, (d_out_max + EXPAND_COLS - 1) / EXPAND_COLS), SG_THREADS, expand_smem, st>>>(a);
+  const dim3 egrid(tiles * a.n_mats, (d_out_max + EXPAND_COLS - 1) / EXPAND_COLS);
+  if (a.all_segments) sgmv_expand_kernel<TM, RMAX, true><<<egrid, SG_THREADS, expand_smem, st>>>(a);
+  else sgmv_expand_kernel<TM, RMAX, false><<<egrid, SG_THREADS, expand_smem, st>>>(a);
   FL_CUDA(p, cudaGetLastError());
   return FL_OK;
 }
@@ -510,9 +592,22 @@ size_t fl_lora_sgmv_workspace(int n_tokens, int n_mats) {
   return (size_t)n_mats * pick_ksplit(n_tokens) * (size_t)n_tokens * FL_MAX_RANK * sizeof(float) + 256;
 }
 
-int fl_lora_sgmv_multi(fl_pool* p, fl_bf16* const* ys, const fl_bf16* x, const int* mat_indices, int n_mats,
-                       const int32_t* seg_indptr, const int32_t* lora_ids, int n_seg, int n_tokens,
-                       float scale, void* workspace, size_t workspace_bytes, fl_stream stream) {
+}  // extern "C"
+
+namespace {
+
+struct KvDest {      // where K and V results go when they are appended to the pool by the projection itself
+  int k_slot, v_slot;           // positions of the K and V projections in the call's list
+  const int32_t* req_indptr;
+  const int32_t* tbl_indptr;
+  const uint32_t* tbl;
+  const int32_t* prefix_lens;
+  int n_req, n_kv;
+};
+
+int sgmv_common(fl_pool* p, fl_bf16* const* ys, const fl_bf16* x, const int* mat_indices, int n_mats,
+                const int32_t* seg_indptr, const int32_t* lora_ids, int n_seg, int n_tokens,
+                float scale, void* workspace, size_t workspace_bytes, fl_stream stream, const KvDest* kv) {
   if (!p || n_mats < 1 || n_mats > FL_MAX_MATS || n_seg < 0 || n_tokens < 0 || !ys || !mat_indices) return FL_EINVAL;
   if (n_seg == 0 || n_tokens == 0) return FL_OK;
   if (!x || !seg_indptr || !lora_ids || !workspace) return FL_EINVAL;
@@ -528,6 +623,32 @@ int fl_lora_sgmv_multi(fl_pool* p, fl_bf16* const* ys, const fl_bf16* x, const i
     a.y[j] = reinterpret_cast<__nv_bfloat16*>(ys[j]);
     a.mat_index[j] = mi;
     d_out_max = d_out_max > p->mats[mi].d_out ? d_out_max : p->mats[mi].d_out;
+  }
+  for (int j = 0; j < FL_MAX_MATS; ++j) {
+    a.kv_side[j] = -1;
+    a.d_out[j] = j < n_mats ? p->mats[mat_indices[j]].d_out : 0;
+  }
+  a.all_segments = 0;
+  a.req_indptr = a.tbl_indptr = a.prefix_lens = nullptr;
+  a.tbl = nullptr;
+  a.n_req = a.n_kv = a.bt = 0;
+  if (kv) {
+    const size_t per_tok = (size_t)2 * kv->n_kv * FL_HEAD_DIM * 2;
+    if (kv->n_kv < 1 || kv->n_req < 1 || p->block_bytes % per_tok != 0 || kv->k_slot == kv->v_slot) return FL_EINVAL;
+    if (!kv->req_indptr || !kv->tbl_indptr || !kv->tbl || !kv->prefix_lens) return FL_EINVAL;
+    for (int side = 0; side < 2; ++side) {
+      const int slot = side ? kv->v_slot : kv->k_slot;
+      if (slot < 0 || slot >= n_mats || a.d_out[slot] != kv->n_kv * FL_HEAD_DIM) return FL_EINVAL;
+      a.kv_side[slot] = side;
+    }
+    a.all_segments = 1;
+    a.req_indptr = kv->req_indptr;
+    a.tbl_indptr = kv->tbl_indptr;
+    a.tbl = kv->tbl;
+    a.prefix_lens = kv->prefix_lens;
+    a.n_req = kv->n_req;
+    a.n_kv = kv->n_kv;
+    a.bt = (int)(p->block_bytes / per_tok);
   }
   a.n_mats = n_mats;
   a.seg_indptr = seg_indptr;
@@ -558,6 +679,28 @@ int fl_lora_sgmv_multi(fl_pool* p, fl_bf16* const* ys, const fl_bf16* x, const i
   }
   if (prev != p->device && prev >= 0) cudaSetDevice(prev);
   return rc;
+}
+
+}  // namespace
+
+extern "C" {
+
+int fl_lora_sgmv_multi(fl_pool* p, fl_bf16* const* ys, const fl_bf16* x, const int* mat_indices, int n_mats,
+                       const int32_t* seg_indptr, const int32_t* lora_ids, int n_seg, int n_tokens,
+                       float scale, void* workspace, size_t workspace_bytes, fl_stream stream) {
+  return sgmv_common(p, ys, x, mat_indices, n_mats, seg_indptr, lora_ids, n_seg, n_tokens, scale, workspace,
+                     workspace_bytes, stream, nullptr);
+}
+
+int fl_lora_sgmv_qkv_append(fl_pool* p, fl_bf16* y_q, const fl_bf16* y_k, const fl_bf16* y_v, const fl_bf16* x,
+                            int mat_q, int mat_k, int mat_v, const int32_t* seg_indptr, const int32_t* lora_ids,
+                            int n_seg, int n_tokens, float scale, const int32_t* req_indptr,
+                            const int32_t* kv_tbl_indptr, const uint32_t* kv_tbl, const int32_t* prefix_lens,
+                            int n_req, int n_kv_heads, void* workspace, size_t workspace_bytes, fl_stream stream) {
+  fl_bf16* ys[3] = {y_q, const_cast<fl_bf16*>(y_k), const_cast<fl_bf16*>(y_v)};
+  const int mi[3] = {mat_q, mat_k, mat_v};
+  const KvDest kv = {1, 2, req_indptr, kv_tbl_indptr, kv_tbl, prefix_lens, n_req, n_kv_heads};
+  return sgmv_common(p, ys, x, mi, 3, seg_indptr, lora_ids, n_seg, n_tokens, scale, workspace, workspace_bytes, stream, &kv);
 }
 
 int fl_lora_sgmv(fl_pool* p, fl_bf16* y, const fl_bf16* x, int mat_index,

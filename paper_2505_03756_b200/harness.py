@@ -178,6 +178,16 @@ class Session:
             fl.fl_lora_sgmv_multi(self.pool, ys, x, [self.mat_index[m] for m in mats], self.t_seg_indptr,
                                   self.t_seg_lora, self.n_seg, T, scale, ws, stream)
 
+    def sgmv_qkv_append(self, y_q, y_k, y_v, x, scale=None, stream=None):
+        """q += LoRA term in place; base k, v + LoRA term written straight into the batch's pool blocks."""
+        T = self.wl.n_tokens
+        ws = self.workspace("sgmv", fl.fl_lora_sgmv_workspace(T, 3))
+        scale = self.wl.scale if scale is None else scale
+        fl.fl_lora_sgmv_qkv_append(self.pool, y_q, y_k, y_v, x, self.mat_index["q"], self.mat_index["k"],
+                                   self.mat_index["v"], self.t_seg_indptr, self.t_seg_lora, self.n_seg, T, scale,
+                                   self.t_req_indptr, self.t_tbl_indptr, self.t_tbl, self.t_prefix, self.wl.n_req,
+                                   self.shape.n_kv_heads, ws, stream)
+
     def kv_append(self, k_new, v_new, stream=None):
         fl.fl_kv_append(self.pool, k_new, v_new, self.t_req_indptr, self.t_tbl_indptr, self.t_tbl, self.t_prefix,
                         self.wl.n_req, self.wl.n_tokens, self.shape.n_kv_heads, stream)

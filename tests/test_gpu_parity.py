@@ -425,3 +425,50 @@ def test_layer_step_replayed_from_cuda_graph_is_bit_identical(H):
         assert s.status()["device_flags"] == 0
     finally:
         s.close()
+
+
+# ------------------------------------------------------------------ q/k/v projection with the KV store folded in
+@pytest.mark.parametrize("name", ["tiny", "prefill7b", "decode13b", "gqa34b", "swapstress"])
+def test_sgmv_qkv_append_equals_projection_then_append(H, name):
+    from paper_2505_03756_b200 import binding as fl
+    wl = synth.make_workload(name, **REDUCED[name])
+    s = _session(H, wl)
+    try:
+        s.fill_prefix_kv()
+        sh, T = wl.shape, wl.n_tokens
+        tx = H.f32_to_dev(wl.x("q"), s.dev)
+        seg, ids = wl.segments()
+        for drop_some in (False, True):           # second pass: every other segment has no adapter (base K/V only)
+            lora = s.t_seg_lora
+            if drop_some:
+                mixed = ids.copy()
+                mixed[::2] = -1
+                lora = torch.from_numpy(mixed).to(s.dev)
+            tables = [[int(b) for b in t] for t in s.kv_tables]
+            blocks = sorted({b for t in tables for b in t})
+            # reference: the two calls
+            ty = {m: H.f32_to_dev(wl.y_base(m), s.dev) for m in "qkv"}
+            ws = s.workspace("sgmv", fl.fl_lora_sgmv_workspace(T, 3))
+            fl.fl_lora_sgmv_multi(s.pool, [ty["q"], ty["k"], ty["v"]], tx, [s.mat_index[m] for m in "qkv"], s.t_seg_indptr,
+                                  lora, s.n_seg, T, wl.scale, ws)
+            s.kv_append(ty["k"], ty["v"])
+            torch.cuda.synchronize()
+            want_q = ty["q"].clone()
+            want_blocks = fl.device_block_bytes(s.pool, s.block_bytes, blocks)
+            # scribble over the new tokens' slots so that a missing write shows
+            junk = torch.full_like(ty["k"], 7.0)
+            s.kv_append(junk, junk)
+            # the fused call
+            tz = {m: H.f32_to_dev(wl.y_base(m), s.dev) for m in "qkv"}
+            fl.fl_lora_sgmv_qkv_append(s.pool, tz["q"], tz["k"], tz["v"], tx, s.mat_index["q"], s.mat_index["k"],
+                                       s.mat_index["v"], s.t_seg_indptr, lora, s.n_seg, T, wl.scale, s.t_req_indptr,
+                                       s.t_tbl_indptr, s.t_tbl, s.t_prefix, wl.n_req, sh.n_kv_heads, ws)
+            torch.cuda.synchronize()
+            assert s.status()["device_flags"] == 0
+            assert torch.equal(tz["q"], want_q)
+            got_blocks = fl.device_block_bytes(s.pool, s.block_bytes, blocks)
+            assert np.array_equal(got_blocks, want_blocks), (name, drop_some)
+            # k, v inputs are left as they were
+            assert np.array_equal(H.dev_to_f32(tz["k"]), wl.y_base("k")) and np.array_equal(H.dev_to_f32(tz["v"]), wl.y_base("v"))
+    finally:
+        s.close()

@@ -4,10 +4,12 @@
 // Two kernels.  shrink: v = x A_i for a tile of tokens of one segment and a slice of d_in, adapter
 // rows fetched through the adapter's block table with 16-byte cp.async, bf16 mma.sync with fp32
 // accumulation, partial sums written to scratch [mat][k-slice][token][RMAX].  expand: sums the
-// partials, scales, splits v into bf16 hi + lo parts (so the second contraction keeps fp32-level
-// accuracy), multiplies by the B rows of a column range and adds into y with coalesced 16-byte
-// read-modify-write staged through shared memory.  Both are bound by HBM traffic (x and y rows
-// for long segments, adapter rows for decode-sized segments), not by the contraction.
+// partials, scales, rounds v to bf16, multiplies by the B rows of a column range (fp32 accumulation),
+// rounds that LoRA term to bf16 into a tile of its own and adds it to the staged y rows with packed
+// bf16 adds while the rows go out as coalesced 16-byte stores: y_out = rn(y + rn(term)).  The term is a
+// small correction of y, so its own 2^-9 roundings stay far below y's final rounding.  Both kernels are
+// bound by memory traffic (x and y rows for long segments, adapter rows for decode-sized segments) and by
+// the instructions spent per byte, not by the contraction.
 #include "mma_utils.cuh"
 #include "pool.cuh"
 
@@ -79,6 +81,17 @@ __device__ __forceinline__ bool find_tile(const int32_t* __restrict__ seg_indptr
     base += total;
   }
   return false;
+}
+
+// Eight bf16 sums (round to nearest even each) of two 16-byte chunks.
+__device__ __forceinline__ uint4 add_bf16x8(uint4 a, uint4 b) {
+  uint4 r;
+  const __nv_bfloat162* pa = reinterpret_cast<const __nv_bfloat162*>(&a);
+  const __nv_bfloat162* pb = reinterpret_cast<const __nv_bfloat162*>(&b);
+  __nv_bfloat162* pr = reinterpret_cast<__nv_bfloat162*>(&r);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) pr[i] = __hadd2(pa[i], pb[i]);
+  return r;
 }
 
 // Start of rank-row `row` of a stream (class table entry tab, first row row0, rows per block rpb, row width).
@@ -375,8 +388,8 @@ __global__ void __launch_bounds__(SG_THREADS, expand_min_ctas(TM, RMAX, KV)) sgm
   const int warp_m = warp % WM, warp_n = warp / WM;
   const int g = lane >> 2, t4 = lane & 3;
 
-  // v fragments: sum of the k-slices, scaled, as bf16 hi + lo
-  uint32_t ahi[RMAX / 16][4], alo[RMAX / 16][4];
+  // v fragments: sum of the k-slices, scaled, rounded to bf16
+  uint32_t av[RMAX / 16][4];
   {
     const int r0 = tok0 + warp_m * 16 + g, r1 = r0 + 8;
 #pragma unroll
@@ -394,9 +407,7 @@ __global__ void __launch_bounds__(SG_THREADS, expand_min_ctas(TM, RMAX, KV)) sgm
           }
         }
         s.x *= a.scale; s.y *= a.scale;
-        const __nv_bfloat16 hx = __float2bfloat16_rn(s.x), hy = __float2bfloat16_rn(s.y);
-        ahi[ks][q] = pack_bf16(__bfloat162float(hx), __bfloat162float(hy));
-        alo[ks][q] = pack_bf16(s.x - __bfloat162float(hx), s.y - __bfloat162float(hy));
+        av[ks][q] = pack_bf16(s.x, s.y);
       }
     }
   }
@@ -492,23 +503,20 @@ __global__ void __launch_bounds__(SG_THREADS, expand_min_ctas(TM, RMAX, KV)) sgm
           uint32_t bf[4];
           ldmatrix_x4_trans(bf, bs + swz(16 * ks + (lane & 7) + 8 * ((lane >> 3) & 1),
                                          warp_n * NTW + 2 * p + (lane >> 4), 16));
-          mma_bf16(acc[2 * p], ahi[ks], bf[0], bf[1]);
-          mma_bf16(acc[2 * p], alo[ks], bf[0], bf[1]);
-          mma_bf16(acc[2 * p + 1], ahi[ks], bf[2], bf[3]);
-          mma_bf16(acc[2 * p + 1], alo[ks], bf[2], bf[3]);
+          mma_bf16(acc[2 * p], av[ks], bf[0], bf[1]);
+          mma_bf16(acc[2 * p + 1], av[ks], bf[2], bf[3]);
         }
       }
     }
-    // add into the staged y rows (each element is owned by exactly one thread)
+    // the LoRA term of this sub-tile as bf16 pairs into its own tile (each element is owned by exactly one thread)
+    unsigned char* dsm = smem + 2 * STAGE_BYTES;
 #pragma unroll
     for (int n = 0; n < NTW; ++n) {
       const int chunk = warp_n * NTW + n;
 #pragma unroll
       for (int h = 0; h < 2; ++h) {
         const int row = warp_m * 16 + g + 8 * h;
-        uint32_t* p = reinterpret_cast<uint32_t*>(ysm + swz(row, chunk, 16) + 4 * t4);
-        const float2 old = unpack_bf16(*p);
-        *p = pack_bf16(old.x + acc[n][2 * h], old.y + acc[n][2 * h + 1]);
+        *reinterpret_cast<uint32_t*>(dsm + swz(row, chunk, 16) + 4 * t4) = pack_bf16(acc[n][2 * h], acc[n][2 * h + 1]);
       }
     }
     __syncthreads();
@@ -519,7 +527,8 @@ __global__ void __launch_bounds__(SG_THREADS, expand_min_ctas(TM, RMAX, KV)) sgm
 #pragma unroll
           for (int i = 0; i < YR; ++i)
             if (yok[i])
-              *reinterpret_cast<uint4*>(yrow[i] + col) = *reinterpret_cast<const uint4*>(ysm + swz(crow + 8 * i, cchunk, 16));
+              *reinterpret_cast<uint4*>(yrow[i] + col) = add_bf16x8(*reinterpret_cast<const uint4*>(ysm + swz(crow + 8 * i, cchunk, 16)),
+                                                                    *reinterpret_cast<const uint4*>(dsm + swz(crow + 8 * i, cchunk, 16)));
         } else if (KV) {
           // a sub-tile is one KV head: [K|V][head][slot][128] inside the block
           static_assert(NSUB == FL_HEAD_DIM, "a sub-tile must be one head");
@@ -530,7 +539,8 @@ __global__ void __launch_bounds__(SG_THREADS, expand_min_ctas(TM, RMAX, KV)) sgm
               const uint32_t loc = kvloc[KV ? i : 0];
               const int slot = (loc >> 1) & 15;
               unsigned char* dst = a.pv.slab + (size_t)(loc >> 5) * a.pv.block_bytes + head_off + slot * (FL_HEAD_DIM * 2);
-              *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(ysm + swz(crow + 8 * i, cchunk, 16));
+              *reinterpret_cast<uint4*>(dst) = add_bf16x8(*reinterpret_cast<const uint4*>(ysm + swz(crow + 8 * i, cchunk, 16)),
+                                                          *reinterpret_cast<const uint4*>(dsm + swz(crow + 8 * i, cchunk, 16)));
               if (side == 1 && (loc & 1u))     // V of a request's last token: clear the slots behind it
                 for (int z = slot + 1; z < a.bt; ++z)
                   *reinterpret_cast<uint4*>(dst + (z - slot) * (FL_HEAD_DIM * 2)) = make_uint4(0u, 0u, 0u, 0u);
@@ -556,7 +566,7 @@ template <int TM, int RMAX>
 int launch_pair(fl_pool* p, const SgmvArgs& a, int tiles, int d_out_max, cudaStream_t st) {
   static bool configured[16] = {};
   const int shrink_smem = SH_STAGES * (TM + RMAX) * 128;
-  const int expand_smem = 2 * (TM + RMAX) * 256;
+  const int expand_smem = 2 * (TM + RMAX) * 256 + TM * 256;     // two stages of (y, B) + the LoRA-term tile
   if (!configured[p->device & 15]) {
     FL_CUDA(p, cudaFuncSetAttribute(sgmv_shrink_kernel<TM, RMAX>, cudaFuncAttributeMaxDynamicSharedMemorySize, shrink_smem));
     FL_CUDA(p, cudaFuncSetAttribute(sgmv_expand_kernel<TM, RMAX, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, expand_smem));

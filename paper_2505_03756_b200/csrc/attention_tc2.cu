@@ -151,67 +151,74 @@ attn_prefill_tc2_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap kv
   // warpgroup does not need
   if (warp >= 8) {
     asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
-    if (warp == 8 && lane == 0) {
+    if (warp == 8) {
       // ------------------------------------------------ unit fetch + TMA producer
+      // The whole warp runs the loop; lane 0 fetches units and does the waiting, lanes 0-7 each own one of a
+      // tile's eight pages (their block-id loads and their TMA issues run side by side).
       int fill = 0;                    // ring fills so far, over all units
       int n_valid = 0;                 // units whose Q tiles were loaded so far
-      for (int k = 0;; ++k) {
-        if (k >= 2 && !mbar_wait(bar(C_UEMPTY + (k & 1)), ((k >> 1) - 1) & 1, abort_flag)) break;
-        const int u = k == 0 ? (int)blockIdx.x : (int)gridDim.x + atomicAdd(&a.hdr->next_unit, 1);
-        Unit t;
-        if (u < n_units) t = decode_unit(a, u, heads_per_item);
-        else t.index = -1;
-        unit_slot[k & 1] = t;
-        mbar_arrive(bar(C_UFULL + (k & 1)));
-        if (t.index < 0) break;
-        if (!t.valid) {
-          atomicOr(a.pv.flags, (uint32_t)FLAG_BAD_POS);
+      bool ok = true;
+      for (int k = 0; ok; ++k) {
+        if (lane == 0) {
+          Unit t;
+          t.index = -1;
+          t.valid = 0;
+          if (k < 2 || mbar_wait(bar(C_UEMPTY + (k & 1)), ((k >> 1) - 1) & 1, abort_flag)) {
+            const int u = k == 0 ? (int)blockIdx.x : (int)gridDim.x + atomicAdd(&a.hdr->next_unit, 1);
+            if (u < n_units) t = decode_unit(a, u, heads_per_item);
+          }
+          unit_slot[k & 1] = t;
+          mbar_arrive(bar(C_UFULL + (k & 1)));
+        }
+        __syncwarp();
+        const Unit* up = unit_slot + (k & 1);
+        if (up->index < 0) break;
+        if (!up->valid) {
+          if (lane == 0) atomicOr(a.pv.flags, (uint32_t)FLAG_BAD_POS);
           continue;
         }
+        const int n_kt_max = up->n_kt_max, n_pages = up->n_pages, tbl0 = up->tbl0, h = up->h;
+        const int rows_b = up->rows[1];
         // Q buffers are free once the previous unit's last S MMA has completed
-        if (n_valid > 0 && !mbar_wait(bar(C_QEMPTY), (n_valid - 1) & 1, abort_flag)) break;
-        ++n_valid;
-        mbar_expect_tx(bar(C_QFULL), t.rows[1] > 0 ? 2 * TILE_BYTES : TILE_BYTES);
-#pragma unroll
-        for (int x = 0; x < 2; ++x) {
-          if (t.rows[x] > 0) {
-            tma_load_3d(sbase + OFF_Q2 + x * TILE_BYTES, &q_map, bar(C_QFULL), 0, t.hq[x], t.tok0[x]);
-            tma_load_3d(sbase + OFF_Q2 + x * TILE_BYTES + HALF_BYTES, &q_map, bar(C_QFULL), 64, t.hq[x], t.tok0[x]);
-          }
+        if (lane == 0) {
+          if (n_valid > 0) ok = mbar_wait(bar(C_QEMPTY), (n_valid - 1) & 1, abort_flag);
+          if (ok) mbar_expect_tx(bar(C_QFULL), rows_b > 0 ? 2 * TILE_BYTES : TILE_BYTES);
         }
-        bool ok = true;
-        for (int j = 0; ok && j < t.n_kt_max; ++j) {
-          // the tile's eight block ids first (independent loads, in flight together, before any wait); K_j and
-          // V_j come from the same blocks
-          uint32_t blk[KT2 / BT];
-#pragma unroll
-          for (int pg = 0; pg < KT2 / BT; ++pg)   // pages behind the last needed key are masked anyway: re-read the last valid page
-            blk[pg] = a.tbl[t.tbl0 + min(j * (KT2 / BT) + pg, t.n_pages - 1)];
-          bool bad = false;
-#pragma unroll
-          for (int pg = 0; pg < KT2 / BT; ++pg) {
-            if (blk[pg] >= a.pv.n_blocks) {
-              bad = true;
-              blk[pg] = 0;
+        ++n_valid;
+        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+        if (!ok) break;
+        if (lane < 4 && (lane < 2 || rows_b > 0)) {          // lane = 2 * tile + half
+          const int x = lane >> 1, half = lane & 1;
+          tma_load_3d(sbase + OFF_Q2 + x * TILE_BYTES + half * HALF_BYTES, &q_map, bar(C_QFULL), 64 * half, up->hq[x], up->tok0[x]);
+        }
+        for (int j = 0; ok && j < n_kt_max; ++j) {
+          // this lane's page of the tile (pages behind the last needed key are masked anyway: re-read the last
+          // valid page); K_j and V_j come from the same blocks
+          uint32_t blk = 0;
+          if (lane < KT2 / BT) {
+            blk = a.tbl[tbl0 + min(j * (KT2 / BT) + lane, n_pages - 1)];
+            if (blk >= a.pv.n_blocks) {
+              atomicOr(a.pv.flags, (uint32_t)FLAG_BAD_BLOCK);
+              blk = 0;
             }
           }
-          if (bad) atomicOr(a.pv.flags, (uint32_t)FLAG_BAD_BLOCK);
 #pragma unroll
           for (int side = 0; side < 2; ++side, ++fill) {
             const int s = fill % NSLOT, use = fill / NSLOT;
-            if (use > 0 && !mbar_wait(bar(C_EMPTY + s), (use - 1) & 1, abort_flag)) { ok = false; break; }
-            mbar_expect_tx(bar(C_FULL + s), TILE_BYTES);
-            const uint32_t dst = sbase + OFF_RING + s * TILE_BYTES;
-            const int slot_head = side * a.n_kv + t.h;
-#pragma unroll
-            for (int pg = 0; pg < KT2 / BT; ++pg) {
-              const uint32_t off = pg * (BT * 128);
-              tma_load_4d(dst + off, &kv_map, bar(C_FULL + s), 0, 0, slot_head, (int)blk[pg]);
-              tma_load_4d(dst + HALF_BYTES + off, &kv_map, bar(C_FULL + s), 64, 0, slot_head, (int)blk[pg]);
+            if (lane == 0) {
+              if (use > 0) ok = mbar_wait(bar(C_EMPTY + s), (use - 1) & 1, abort_flag);
+              if (ok) mbar_expect_tx(bar(C_FULL + s), TILE_BYTES);
+            }
+            ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;     // the transaction count is armed before any copy is issued
+            if (!ok) break;
+            if (lane < KT2 / BT) {
+              const uint32_t dst = sbase + OFF_RING + s * TILE_BYTES + lane * (BT * 128);
+              const int slot_head = side * a.n_kv + h;
+              tma_load_4d(dst, &kv_map, bar(C_FULL + s), 0, 0, slot_head, (int)blk);
+              tma_load_4d(dst + HALF_BYTES, &kv_map, bar(C_FULL + s), 64, 0, slot_head, (int)blk);
             }
           }
         }
-        if (!ok) break;
       }
     } else if (warp == 9 && lane == 0) {
       // ------------------------------------------------ MMA issuer

@@ -472,3 +472,17 @@ def test_sgmv_qkv_append_equals_projection_then_append(H, name):
             assert np.array_equal(H.dev_to_f32(tz["k"]), wl.y_base("k")) and np.array_equal(H.dev_to_f32(tz["v"]), wl.y_base("v"))
     finally:
         s.close()
+
+
+@pytest.mark.parametrize("heads", [(6, 2), (64, 2), (5, 5)])
+def test_attention_unusual_head_groupings(H, heads):
+    # odd group sizes take the one-head-per-unit path of the tensor-core kernel; a group wider than the decode
+    # kernel's 16 rows sends even one-token requests through the prefill kernel
+    n_q, n_kv = heads
+    sh = synth.LayerShape(n_q * 128, n_q, n_kv)
+    wl = synth.make_workload("tiny", n_req=4, len_range=(0, 0), n_adapters=1, shape=sh)
+    wl.prefix_lens[:] = [200, 0, 33, 500]
+    wl.new_lens[:] = [1, 140, 300, 2]
+    wl.pool_blocks = 160
+    for kernel in (0, 1):
+        _attention_case(H, wl, prefill_kernel=kernel)

@@ -355,6 +355,10 @@ __global__ void __launch_bounds__(SG_THREADS) sgmv_shrink3_kernel(const SgmvArgs
 // than a few spilled values)
 constexpr int expand_min_ctas(int tm, int rmax, bool) { return tm == 16 ? 5 : (rmax == 16 ? 4 : 3); }
 
+// whether the LoRA-term tile reuses the adapter-row buffer of the stage (it has to fit there)
+__host__ __device__ constexpr bool expand_alias(int tm, int rmax) { return rmax >= 64 && rmax >= tm; }
+constexpr int expand_smem_bytes(int tm, int rmax) { return 2 * (tm + rmax) * 256 + (expand_alias(tm, rmax) ? 0 : tm * 256); }
+
 template <int TM, int RMAX, bool KV>
 __global__ void __launch_bounds__(SG_THREADS, expand_min_ctas(TM, RMAX, KV)) sgmv_expand_kernel(const SgmvArgs a) {
   extern __shared__ __align__(128) unsigned char smem[];
@@ -508,8 +512,12 @@ __global__ void __launch_bounds__(SG_THREADS, expand_min_ctas(TM, RMAX, KV)) sgm
         }
       }
     }
-    // the LoRA term of this sub-tile as bf16 pairs into its own tile (each element is owned by exactly one thread)
-    unsigned char* dsm = smem + 2 * STAGE_BYTES;
+    // the LoRA term of this sub-tile as bf16 pairs into a tile of its own (each element is owned by exactly one
+    // thread); at rank 64 that tile takes the place of the adapter rows the MMAs have just consumed, which brings
+    // the CTA to 64 KB and a third CTA onto the SM
+    constexpr bool ALIAS = expand_alias(TM, RMAX);
+    unsigned char* dsm = ALIAS ? smem + st * STAGE_BYTES + TM * 256 : smem + 2 * STAGE_BYTES;
+    if (ALIAS) __syncthreads();
 #pragma unroll
     for (int n = 0; n < NTW; ++n) {
       const int chunk = warp_n * NTW + n;
@@ -566,7 +574,7 @@ template <int TM, int RMAX>
 int launch_pair(fl_pool* p, const SgmvArgs& a, int tiles, int d_out_max, cudaStream_t st) {
   static bool configured[16] = {};
   const int shrink_smem = SH_STAGES * (TM + RMAX) * 128;
-  const int expand_smem = 2 * (TM + RMAX) * 256 + TM * 256;     // two stages of (y, B) + the LoRA-term tile
+  const int expand_smem = expand_smem_bytes(TM, RMAX);     // two stages of (y, B) + the LoRA-term tile
   if (!configured[p->device & 15]) {
     FL_CUDA(p, cudaFuncSetAttribute(sgmv_shrink_kernel<TM, RMAX>, cudaFuncAttributeMaxDynamicSharedMemorySize, shrink_smem));
     FL_CUDA(p, cudaFuncSetAttribute(sgmv_expand_kernel<TM, RMAX, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, expand_smem));

@@ -19,7 +19,7 @@ constexpr int SG_THREADS = 128;
 constexpr int KS = 64;            // d_in elements per shrink pipeline stage (128-byte rows)
 constexpr int SH_STAGES = 4;
 constexpr int NSUB = 128;         // y columns per expand sub-tile (256-byte rows)
-constexpr int EXPAND_COLS = 512;  // y columns per expand CTA
+constexpr int EXPAND_COLS_MIN = 512, EXPAND_COLS_MAX = 4096;   // y columns per expand CTA: picked per call
 constexpr int KSPLIT_MAX = 8;
 
 struct SgmvArgs {
@@ -34,6 +34,7 @@ struct SgmvArgs {
   float scale;
   float* v;        // [n_mats][ksplit][n_tokens][RMAX]
   int ksplit;
+  int expand_cols;   // y columns one expand CTA covers
   int d_out[FL_MAX_MATS];
   // K / V projections whose result goes straight into the requests' pool blocks instead of back into y
   // (kv_side[j] = 0: K, 1: V, -1: y updated in place); then segments without an adapter are tiled too
@@ -382,9 +383,9 @@ __global__ void __launch_bounds__(SG_THREADS, expand_min_ctas(TM, RMAX, KV)) sgm
     return;                                // no adapter and y stays where it is: nothing to do
   }
   const int d_out = a.d_out[j];
-  const int c0 = blockIdx.y * EXPAND_COLS;
+  const int c0 = blockIdx.y * a.expand_cols;
   if (c0 >= d_out) return;
-  const int c1 = min(d_out, c0 + EXPAND_COLS);
+  const int c1 = min(d_out, c0 + a.expand_cols);
   const int n_sub = (c1 - c0 + NSUB - 1) / NSUB;
 
   constexpr int WM = TM / 16, WN = 4 / WM;     // warps along tokens / along columns
@@ -570,8 +571,22 @@ int pick_ksplit(int n_tokens) {
   return ks;
 }
 
+// Columns per expand CTA.  Every CTA pays a prologue of dependent look-ups (its tile, the adapter's directory
+// entry and row tables, the v fragments, the K/V destinations) that wider CTAs spread over more sub-tiles; the
+// widest slice that still leaves about ten CTAs per SM in the grid wins.
+int pick_expand_cols(const SgmvArgs& a, int tiles) {
+  int cols = EXPAND_COLS_MAX;
+  for (; cols > EXPAND_COLS_MIN; cols /= 2) {
+    long ctas = 0;
+    for (int j = 0; j < a.n_mats; ++j) ctas += (long)tiles * ((a.d_out[j] + cols - 1) / cols);
+    if (ctas >= 1480) break;
+  }
+  return cols;
+}
+
 template <int TM, int RMAX>
-int launch_pair(fl_pool* p, const SgmvArgs& a, int tiles, int d_out_max, cudaStream_t st) {
+int launch_pair(fl_pool* p, SgmvArgs& a, int tiles, int d_out_max, cudaStream_t st) {
+  a.expand_cols = pick_expand_cols(a, tiles);
   static bool configured[16] = {};
   const int shrink_smem = SH_STAGES * (TM + RMAX) * 128;
   const int expand_smem = expand_smem_bytes(TM, RMAX);     // two stages of (y, B) + the LoRA-term tile
@@ -592,7 +607,7 @@ int launch_pair(fl_pool* p, const SgmvArgs& a, int tiles, int d_out_max, cudaStr
   } else {
     sgmv_shrink_kernel<TM, RMAX><<<dim3(tiles * a.n_mats, a.ksplit), SG_THREADS, shrink_smem, st>>>(a);
   }
-  const dim3 egrid(tiles * a.n_mats, (d_out_max + EXPAND_COLS - 1) / EXPAND_COLS);
+  const dim3 egrid(tiles * a.n_mats, (d_out_max + a.expand_cols - 1) / a.expand_cols);
   if (a.all_segments) sgmv_expand_kernel<TM, RMAX, true><<<egrid, SG_THREADS, expand_smem, st>>>(a);
   else sgmv_expand_kernel<TM, RMAX, false><<<egrid, SG_THREADS, expand_smem, st>>>(a);
   FL_CUDA(p, cudaGetLastError());

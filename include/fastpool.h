@@ -235,6 +235,21 @@ int fl_swap_in(fl_pool* pool, const uint32_t* dev_ids, const uint32_t* host_ids,
 int fl_swap_record(fl_pool* pool, fl_event ev, fl_stream side);
 int fl_swap_wait(fl_pool* pool, fl_event ev, int timeout_ms);
 
+/* ---------------------------------------------------------------- readiness while blocks are in flight
+ * Section 4.3 "Asynchronous Swapping-in/out": a query whose adapter or cached KV is still being swapped in
+ * waits, and the queries that are ready run meanwhile.  Host code; all pointers are host pointers.
+ * fl_inflight_mark: the listed device blocks are the targets of copies already enqueued on a side stream;
+ * they count as in flight until `ev` - recorded behind those copies with fl_swap_record - has completed.  The
+ * caller keeps `ev` alive until then.  A block marked again moves to the newer event.  FL_EBADID: id out of range.
+ * fl_requests_ready: request r touches the device blocks blks[blk_indptr[r] .. blk_indptr[r+1]) (its adapter's
+ * blocks and its KV blocks); ready[r] = 1 when none of them is in flight, else 0.  Events are polled first
+ * (cudaEventQuery, no waiting) and finished ones release their blocks.  *n_ready (may be NULL) = how many are
+ * ready.  fl_inflight_count: blocks still waiting for their copies after the same poll. */
+int fl_inflight_mark(fl_pool* pool, const uint32_t* dev_ids, uint32_t n, fl_event ev);
+int fl_requests_ready(fl_pool* pool, const int32_t* blk_indptr, const uint32_t* blks, int n_req, uint8_t* ready,
+                      int* n_ready);
+int fl_inflight_count(fl_pool* pool, uint32_t* n_blocks);
+
 /* ---------------------------------------------------------------- cache swapper (Section 5; host code, no GPU work)
  * Decides WHICH nodes (LoRA adapters, KV caches) move between HBM and host memory; the block lists of
  * the chosen nodes then go to fl_swap_out / fl_swap_in.  A node is described by what the usage

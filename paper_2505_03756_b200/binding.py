@@ -85,6 +85,9 @@ _SIGS = {
     "fl_swap_in": (C.c_int, [_vp, _vp, _vp, C.c_uint32, _vp]),
     "fl_swap_record": (C.c_int, [_vp, _vp, _vp]),
     "fl_swap_wait": (C.c_int, [_vp, _vp, C.c_int]),
+    "fl_inflight_mark": (C.c_int, [_vp, _vp, C.c_uint32, _vp]),
+    "fl_requests_ready": (C.c_int, [_vp, _vp, _vp, C.c_int, _vp, C.POINTER(C.c_int)]),
+    "fl_inflight_count": (C.c_int, [_vp, _u32p]),
     "fl_tree_create": (C.c_int, [C.POINTER(_vp), C.c_int]),
     "fl_tree_destroy": (C.c_int, [_vp]),
     "fl_tree_add_lora": (C.c_int, [_vp, C.c_int32, _vp, C.c_uint32, C.c_int, C.c_double, _i32p]),
@@ -321,6 +324,35 @@ def fl_swap_record(pool, event, side_stream):
 
 def fl_swap_wait(pool, event, timeout_ms):
     return lib.fl_swap_wait(pool, event.cuda_event, timeout_ms)
+
+
+def fl_inflight_mark(pool, dev_ids, event):
+    """The listed device blocks wait for copies that finish when `event` (already recorded) completes."""
+    d, pd = _ids(dev_ids)
+    _check(lib.fl_inflight_mark(pool, pd, len(d), event.cuda_event), "fl_inflight_mark")
+
+
+def fl_requests_ready(pool, block_lists):
+    """block_lists[r] = device blocks request r touches; returns a bool array (True = may run now)."""
+    n = len(block_lists)
+    indptr = np.zeros(n + 1, dtype=np.int32)
+    for r, b in enumerate(block_lists):
+        indptr[r + 1] = indptr[r] + len(b)
+    flat = np.ascontiguousarray(np.concatenate([np.asarray(b, dtype=np.uint32) for b in block_lists])
+                                if indptr[-1] else np.zeros(0, dtype=np.uint32), dtype=np.uint32)
+    ready = np.zeros(max(n, 1), dtype=np.uint8)
+    n_ready = C.c_int(0)
+    _check(lib.fl_requests_ready(pool, indptr.ctypes.data, flat.ctypes.data if flat.size else None, n,
+                                 ready.ctypes.data, C.byref(n_ready)), "fl_requests_ready")
+    out = ready[:n].astype(bool)
+    assert int(out.sum()) == n_ready.value
+    return out
+
+
+def fl_inflight_count(pool):
+    c = C.c_uint32(0)
+    _check(lib.fl_inflight_count(pool, C.byref(c)), "fl_inflight_count")
+    return int(c.value)
 
 
 # ------------------------------------------------------------------ cache swapper (host side)

@@ -72,6 +72,10 @@ struct fl_pool {
   uint32_t stage_blocks = 0;
   cudaEvent_t stage_done[2] = {nullptr, nullptr};   // last use of each staging area
   void* tmap_cache = nullptr;                      // tensor maps of the slab, keyed by KV head count
+  // blocks that copies in flight are still filling: inflight[b] = 1 + index into tickets, 0 = none
+  struct Ticket { cudaEvent_t ev = nullptr; uint32_t n_blocks = 0; bool done = false; };
+  std::vector<uint32_t> inflight;
+  std::vector<Ticket> tickets;
   PoolView view() const { return PoolView{slab, block_bytes, n_blocks, d_dir, dir_cap, d_tables, d_flags}; }
 };
 

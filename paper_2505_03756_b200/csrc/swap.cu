@@ -210,6 +210,96 @@ int fl_swap_wait(fl_pool* p, fl_event ev, int timeout_ms) {
   }
 }
 
+// ---- which requests may run while swap-ins are in flight (Section 4.3)
+namespace {
+// Polls the events of the live tickets; a finished ticket releases its blocks lazily (when they are looked at).
+int poll_tickets(fl_pool* p) {
+  for (auto& t : p->tickets) {
+    if (t.n_blocks == 0 || t.done) continue;
+    const cudaError_t e = cudaEventQuery(t.ev);
+    if (e == cudaSuccess) {
+      t.done = true;
+    } else if (e != cudaErrorNotReady) {
+      p->last_cuda = (int)e;
+      return FL_ECUDA;
+    }
+  }
+  return FL_OK;
+}
+// True while block b waits for a copy; clears the mark of a block whose ticket has finished.
+bool block_in_flight(fl_pool* p, uint32_t b) {
+  const uint32_t m = p->inflight[b];
+  if (m == 0) return false;
+  fl_pool::Ticket& t = p->tickets[m - 1];
+  if (!t.done) return true;
+  p->inflight[b] = 0;
+  if (--t.n_blocks == 0) { t.ev = nullptr; t.done = false; }
+  return false;
+}
+}  // namespace
+
+int fl_inflight_mark(fl_pool* p, const uint32_t* dev_ids, uint32_t n, fl_event ev) {
+  if (!p || !ev || (n && !dev_ids)) return FL_EINVAL;
+  for (uint32_t k = 0; k < n; ++k)
+    if (dev_ids[k] >= p->n_blocks) return FL_EBADID;
+  if (n == 0) return FL_OK;
+  if (p->inflight.empty()) p->inflight.assign(p->n_blocks, 0u);
+  uint32_t slot = 0;
+  while (slot < p->tickets.size() && p->tickets[slot].n_blocks != 0) ++slot;
+  if (slot == p->tickets.size()) p->tickets.emplace_back();
+  fl_pool::Ticket& t = p->tickets[slot];
+  t.ev = (cudaEvent_t)ev;
+  t.done = false;
+  t.n_blocks = 0;
+  for (uint32_t k = 0; k < n; ++k) {
+    const uint32_t b = dev_ids[k];
+    const uint32_t old = p->inflight[b];
+    if (old == slot + 1) continue;                    // listed twice in this call
+    if (old != 0) {                                   // a newer copy supersedes the older mark
+      fl_pool::Ticket& o = p->tickets[old - 1];
+      if (--o.n_blocks == 0) { o.ev = nullptr; o.done = false; }
+    }
+    p->inflight[b] = slot + 1;
+    ++t.n_blocks;
+  }
+  return FL_OK;
+}
+
+int fl_requests_ready(fl_pool* p, const int32_t* blk_indptr, const uint32_t* blks, int n_req, uint8_t* ready,
+                      int* n_ready) {
+  if (!p || n_req < 0 || (n_req && (!blk_indptr || !ready))) return FL_EINVAL;
+  for (int r = 0; r < n_req; ++r) {
+    if (blk_indptr[r + 1] < blk_indptr[r] || blk_indptr[r] < 0) return FL_EINVAL;
+    if (blk_indptr[r + 1] > blk_indptr[r] && !blks) return FL_EINVAL;
+    for (int k = blk_indptr[r]; k < blk_indptr[r + 1]; ++k)
+      if (blks[k] >= p->n_blocks) return FL_EBADID;
+  }
+  const int rc = poll_tickets(p);
+  if (rc != FL_OK) return rc;
+  int count = 0;
+  for (int r = 0; r < n_req; ++r) {
+    bool ok = true;
+    if (!p->inflight.empty())
+      for (int k = blk_indptr[r]; k < blk_indptr[r + 1]; ++k)
+        if (block_in_flight(p, blks[k])) ok = false;   // no early exit: every finished mark it meets is cleared
+    ready[r] = ok ? 1 : 0;
+    count += ok ? 1 : 0;
+  }
+  if (n_ready) *n_ready = count;
+  return FL_OK;
+}
+
+int fl_inflight_count(fl_pool* p, uint32_t* n_blocks) {
+  if (!p || !n_blocks) return FL_EINVAL;
+  const int rc = poll_tickets(p);
+  if (rc != FL_OK) return rc;
+  uint32_t c = 0;
+  for (const auto& t : p->tickets)
+    if (t.n_blocks != 0 && !t.done) c += t.n_blocks;
+  *n_blocks = c;
+  return FL_OK;
+}
+
 int fl_kv_append(fl_pool* p, const fl_bf16* k_new, const fl_bf16* v_new, const int32_t* req_indptr,
                  const int32_t* kv_tbl_indptr, const uint32_t* kv_tbl, const int32_t* prefix_lens,
                  int n_req, int n_tokens, int n_kv_heads, fl_stream stream) {

@@ -84,6 +84,12 @@ __device__ __forceinline__ bool find_tile(const int32_t* __restrict__ seg_indptr
   return false;
 }
 
+// Programmatic dependent launch: the shrink lets the expand's CTAs start early (they run their look-ups and the
+// first loads while shrink CTAs are still finishing); the expand waits here for the whole shrink grid and its
+// writes.  Both are no-ops when the kernels are launched without the attribute.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 // Eight bf16 sums (round to nearest even each) of two 16-byte chunks.
 __device__ __forceinline__ uint4 add_bf16x8(uint4 a, uint4 b) {
   uint4 r;
@@ -112,6 +118,7 @@ __device__ __forceinline__ const unsigned char* lora_row(const PoolView& pv, uin
 template <int TM, int RMAX>
 __global__ void __launch_bounds__(SG_THREADS) sgmv_shrink_kernel(const SgmvArgs a) {
   extern __shared__ __align__(128) unsigned char smem[];
+  pdl_launch_dependents();
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int j = blockIdx.x % a.n_mats;
   const int tile = blockIdx.x / a.n_mats;
@@ -236,6 +243,7 @@ __global__ void __launch_bounds__(SG_THREADS) sgmv_shrink3_kernel(const SgmvArgs
   constexpr int TM = 64, NM = 3;
   constexpr int STAGES = RMAX == 64 ? 3 : 4;
   extern __shared__ __align__(128) unsigned char smem[];
+  pdl_launch_dependents();
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int tile = blockIdx.x, split = blockIdx.y;
   int seg, tok0, tok1;
@@ -393,30 +401,6 @@ __global__ void __launch_bounds__(SG_THREADS, expand_min_ctas(TM, RMAX, KV)) sgm
   const int warp_m = warp % WM, warp_n = warp / WM;
   const int g = lane >> 2, t4 = lane & 3;
 
-  // v fragments: sum of the k-slices, scaled, rounded to bf16
-  uint32_t av[RMAX / 16][4];
-  {
-    const int r0 = tok0 + warp_m * 16 + g, r1 = r0 + 8;
-#pragma unroll
-    for (int ks = 0; ks < RMAX / 16; ++ks) {
-#pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        const int row = (q & 1) ? r1 : r0;
-        const int col = 16 * ks + 2 * t4 + ((q & 2) ? 8 : 0);
-        float2 s = make_float2(0.f, 0.f);
-        if (row < tok1 && col < rank) {
-          for (int sp = 0; sp < a.ksplit; ++sp) {
-            const float2 p = *reinterpret_cast<const float2*>(
-                a.v + ((size_t)(j * a.ksplit + sp) * a.n_tokens + row) * RMAX + col);
-            s.x += p.x; s.y += p.y;
-          }
-        }
-        s.x *= a.scale; s.y *= a.scale;
-        av[ks][q] = pack_bf16(s.x, s.y);
-      }
-    }
-  }
-
   constexpr int YR = TM / 8;       // y rows per thread per sub-tile
   constexpr int BR = RMAX / 8;     // adapter rows per thread per sub-tile
   constexpr int STAGE_BYTES = (TM + RMAX) * 256;
@@ -489,6 +473,32 @@ __global__ void __launch_bounds__(SG_THREADS, expand_min_ctas(TM, RMAX, KV)) sgm
 
   load_sub(0, 0);
   cp_async_commit();
+  // v fragments: sum of the k-slices, scaled, rounded to bf16.  Everything above reads only what was in memory
+  // before the shrink started; v is the shrink's output, so this is where a programmatic dependent launch waits.
+  pdl_wait();
+  uint32_t av[RMAX / 16][4];
+  {
+    const int r0 = tok0 + warp_m * 16 + g, r1 = r0 + 8;
+#pragma unroll
+    for (int ks = 0; ks < RMAX / 16; ++ks) {
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const int row = (q & 1) ? r1 : r0;
+        const int col = 16 * ks + 2 * t4 + ((q & 2) ? 8 : 0);
+        float2 s = make_float2(0.f, 0.f);
+        if (row < tok1 && col < rank) {
+          for (int sp = 0; sp < a.ksplit; ++sp) {
+            const float2 p = *reinterpret_cast<const float2*>(
+                a.v + ((size_t)(j * a.ksplit + sp) * a.n_tokens + row) * RMAX + col);
+            s.x += p.x; s.y += p.y;
+          }
+        }
+        s.x *= a.scale; s.y *= a.scale;
+        av[ks][q] = pack_bf16(s.x, s.y);
+      }
+    }
+  }
+
   for (int sub = 0; sub < n_sub; ++sub) {
     const int st = sub & 1;
     if (sub + 1 < n_sub) load_sub(sub + 1, st ^ 1);
@@ -608,9 +618,20 @@ int launch_pair(fl_pool* p, SgmvArgs& a, int tiles, int d_out_max, cudaStream_t 
     sgmv_shrink_kernel<TM, RMAX><<<dim3(tiles * a.n_mats, a.ksplit), SG_THREADS, shrink_smem, st>>>(a);
   }
   const dim3 egrid(tiles * a.n_mats, (d_out_max + a.expand_cols - 1) / a.expand_cols);
-  if (a.all_segments) sgmv_expand_kernel<TM, RMAX, true><<<egrid, SG_THREADS, expand_smem, st>>>(a);
-  else sgmv_expand_kernel<TM, RMAX, false><<<egrid, SG_THREADS, expand_smem, st>>>(a);
+  // the expand may start while the shrink drains (it waits for the shrink's output inside the kernel)
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = egrid;
+  cfg.blockDim = dim3(SG_THREADS);
+  cfg.dynamicSmemBytes = expand_smem;
+  cfg.stream = st;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
   FL_CUDA(p, cudaGetLastError());
+  if (a.all_segments) FL_CUDA(p, cudaLaunchKernelEx(&cfg, sgmv_expand_kernel<TM, RMAX, true>, a));
+  else FL_CUDA(p, cudaLaunchKernelEx(&cfg, sgmv_expand_kernel<TM, RMAX, false>, a));
   return FL_OK;
 }
 

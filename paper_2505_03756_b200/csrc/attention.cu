@@ -41,6 +41,8 @@ __device__ __forceinline__ int block_excl_scan(int val, int* sh, int& total) {
 
 __global__ void __launch_bounds__(256) attn_plan_kernel(const AttnArgs a, int chunk, int qt) {
   __shared__ int sh[8];
+  pdl_wait();                 // the lists may still be read, and the request arrays written, by the kernel before
+  pdl_launch_dependents();    // the prefill kernel sets itself up (barriers, TMEM) while this single CTA plans
   const int group = a.n_q / a.n_kv;
   int base_p = 0, base_d = 0;
   for (int i0 = 0; i0 < a.n_req; i0 += 256) {
@@ -198,6 +200,7 @@ __device__ __forceinline__ const unsigned char* page_ptr(const PoolView& pv, uin
 // their partial (max, sum, O) through shared memory at the end.
 __global__ void __launch_bounds__(ATT_THREADS) attn_decode_kernel(const AttnArgs a) {
   extern __shared__ __align__(128) unsigned char smem[];
+  pdl_wait();
   const int item = blockIdx.x / a.n_kv, h = blockIdx.x % a.n_kv;
   if (item >= a.hdr->n_decode) return;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -321,6 +324,7 @@ __global__ void __launch_bounds__(ATT_THREADS) attn_decode_kernel(const AttnArgs
 
 // Combines the chunk partials of one (request, KV head): grid = n_req * n_kv.
 __global__ void __launch_bounds__(ATT_THREADS) attn_merge_kernel(const AttnArgs a) {
+  pdl_wait();
   const int i = blockIdx.x / a.n_kv, h = blockIdx.x % a.n_kv;
   const int4 info = a.req_info[i];
   if (!info.z || info.y <= 1) return;
@@ -550,7 +554,14 @@ int fl_paged_attention(fl_pool* p, fl_bf16* out, const fl_bf16* q, const int32_t
     }
     // the tensor-core kernels fold sm_scale into the exponent and take row maxima of raw scores: they need sm_scale > 0
     const int kind = sm_scale > 0.f ? p->prefill_kernel : 1;
-    attn_plan_kernel<<<1, 256, 0, st>>>(a, w.chunk, kind == 0 ? tc2_tile_tokens(n_q_heads, n_kv_heads) : (kind == 2 ? QT_TC : QT_MMA));
+    // every kernel of the call is a programmatic dependent launch: it may start while the one before it drains
+    // and waits inside for that kernel's results
+    if (launch_pdl(attn_plan_kernel, dim3(1), dim3(256), 0, st, a, w.chunk,
+                   kind == 0 ? tc2_tile_tokens(n_q_heads, n_kv_heads) : (kind == 2 ? QT_TC : QT_MMA)) != cudaSuccess) {
+      p->last_cuda = (int)cudaGetLastError();
+      rc = FL_ECUDA;
+      break;
+    }
     if (kind == 0) {
       // upper bound of the plan's tile count: full tiles plus one ragged tile per prefill request, and a
       // request is a prefill only with more than DEC_ROWS / group new tokens
@@ -565,9 +576,9 @@ int fl_paged_attention(fl_pool* p, fl_bf16* out, const fl_bf16* q, const int32_t
     } else {
       attn_prefill_kernel<<<(unsigned)w.max_prefill * n_q_heads, ATT_THREADS, PRE_SMEM, st>>>(a);
     }
-    attn_decode_kernel<<<(unsigned)w.max_decode * n_kv_heads, ATT_THREADS, DEC_SMEM, st>>>(a);
-    attn_merge_kernel<<<(unsigned)n_req * n_kv_heads, ATT_THREADS, 0, st>>>(a);
-    cudaError_t e = cudaGetLastError();
+    cudaError_t e = launch_pdl(attn_decode_kernel, dim3((unsigned)w.max_decode * n_kv_heads), dim3(ATT_THREADS), DEC_SMEM, st, a);
+    if (e == cudaSuccess) e = launch_pdl(attn_merge_kernel, dim3((unsigned)n_req * n_kv_heads), dim3(ATT_THREADS), 0, st, a);
+    if (e == cudaSuccess) e = cudaGetLastError();
     if (e != cudaSuccess) {
       p->last_cuda = (int)e;
       rc = FL_ECUDA;

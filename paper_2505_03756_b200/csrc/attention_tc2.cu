@@ -96,8 +96,6 @@ __global__ void __launch_bounds__(T2_THREADS, 1)
 attn_prefill_tc2_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap kv_map, const __grid_constant__ CUtensorMap q_map,
                         int heads_per_item) {
   extern __shared__ __align__(1024) unsigned char smem[];
-  const int n_units = a.hdr->n_prefill * heads_per_item;
-  if ((int)blockIdx.x >= n_units) return;
   const uint32_t sbase = smem_u32(smem);
   if (sbase & 1023u) {   // the swizzled operand tiles need 1024-byte alignment
     if (threadIdx.x == 0) atomicOr(a.pv.flags, (uint32_t)FLAG_WAIT_GAVE_UP);
@@ -136,6 +134,10 @@ attn_prefill_tc2_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap kv
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
+  // everything above touched only this CTA's shared memory and TMEM; the plan (and q, K, V) are the work of the
+  // kernels before this one
+  pdl_wait();
+  const int n_units = a.hdr->n_prefill * heads_per_item;   // a CTA beyond the last unit finds no work and tears down
 
   // Readers take the k-th unit of this CTA from slot k & 1 (index -1 = no more work) and release the slot.
   auto read_unit = [&](int k, bool arrive) -> Unit {
@@ -442,7 +444,7 @@ int launch_prefill_tc2(fl_pool* p, const AttnArgs& a, int n_tokens, int max_item
   const long long units = (long long)max_items * heads_per_item;
   const unsigned grid = (unsigned)std::min<long long>(units, p->sm_count);
   if (grid == 0) return FL_OK;
-  attn_prefill_tc2_kernel<<<grid, T2_THREADS, T2_SMEM, st>>>(a, *kv, qmap, heads_per_item);
+  FL_CUDA(p, launch_pdl(attn_prefill_tc2_kernel, dim3(grid), dim3(T2_THREADS), T2_SMEM, st, a, *kv, qmap, heads_per_item));
   FL_CUDA(p, cudaGetLastError());
   return FL_OK;
 }

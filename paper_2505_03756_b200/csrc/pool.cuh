@@ -79,6 +79,28 @@ struct fl_pool {
   PoolView view() const { return PoolView{slab, block_bytes, n_blocks, d_dir, dir_cap, d_tables, d_flags}; }
 };
 
+// Programmatic dependent launch.  A kernel launched through launch_pdl may start while the kernel before it on
+// the stream is still running; it calls pdl_wait() before it touches anything that kernel may have written (or
+// may still read), which waits for that whole grid and its memory operations.  A kernel that calls
+// pdl_launch_dependents() lets the next one start once all its CTAs are past that point.  Both instructions do
+// nothing in a kernel launched the ordinary way.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 #define FL_CUDA(pool, call)                                  \
   do {                                                       \
     cudaError_t e__ = (call);                                \

@@ -84,12 +84,6 @@ __device__ __forceinline__ bool find_tile(const int32_t* __restrict__ seg_indptr
   return false;
 }
 
-// Programmatic dependent launch: the shrink lets the expand's CTAs start early (they run their look-ups and the
-// first loads while shrink CTAs are still finishing); the expand waits here for the whole shrink grid and its
-// writes.  Both are no-ops when the kernels are launched without the attribute.
-__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
-__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
-
 // Eight bf16 sums (round to nearest even each) of two 16-byte chunks.
 __device__ __forceinline__ uint4 add_bf16x8(uint4 a, uint4 b) {
   uint4 r;
@@ -118,7 +112,8 @@ __device__ __forceinline__ const unsigned char* lora_row(const PoolView& pv, uin
 template <int TM, int RMAX>
 __global__ void __launch_bounds__(SG_THREADS) sgmv_shrink_kernel(const SgmvArgs a) {
   extern __shared__ __align__(128) unsigned char smem[];
-  pdl_launch_dependents();
+  pdl_wait();                 // x may come from the kernel right before this one
+  pdl_launch_dependents();    // the expand may start its look-ups and first loads while this grid drains
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int j = blockIdx.x % a.n_mats;
   const int tile = blockIdx.x / a.n_mats;
@@ -243,7 +238,8 @@ __global__ void __launch_bounds__(SG_THREADS) sgmv_shrink3_kernel(const SgmvArgs
   constexpr int TM = 64, NM = 3;
   constexpr int STAGES = RMAX == 64 ? 3 : 4;
   extern __shared__ __align__(128) unsigned char smem[];
-  pdl_launch_dependents();
+  pdl_wait();                 // x may come from the kernel right before this one
+  pdl_launch_dependents();    // the expand may start its look-ups and first loads while this grid drains
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int tile = blockIdx.x, split = blockIdx.y;
   int seg, tok0, tok1;
@@ -613,25 +609,15 @@ int launch_pair(fl_pool* p, SgmvArgs& a, int tiles, int d_out_max, cudaStream_t 
       FL_CUDA(p, cudaFuncSetAttribute(sgmv_shrink3_kernel<RMAX>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem3));
       configured3[p->device & 15] = true;
     }
-    sgmv_shrink3_kernel<RMAX><<<dim3(tiles, a.ksplit), SG_THREADS, smem3, st>>>(a);
+    FL_CUDA(p, launch_pdl(sgmv_shrink3_kernel<RMAX>, dim3(tiles, a.ksplit), dim3(SG_THREADS), smem3, st, a));
   } else {
-    sgmv_shrink_kernel<TM, RMAX><<<dim3(tiles * a.n_mats, a.ksplit), SG_THREADS, shrink_smem, st>>>(a);
+    FL_CUDA(p, launch_pdl(sgmv_shrink_kernel<TM, RMAX>, dim3(tiles * a.n_mats, a.ksplit), dim3(SG_THREADS), shrink_smem, st, a));
   }
   const dim3 egrid(tiles * a.n_mats, (d_out_max + a.expand_cols - 1) / a.expand_cols);
   // the expand may start while the shrink drains (it waits for the shrink's output inside the kernel)
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[0].val.programmaticStreamSerializationAllowed = 1;
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = egrid;
-  cfg.blockDim = dim3(SG_THREADS);
-  cfg.dynamicSmemBytes = expand_smem;
-  cfg.stream = st;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
   FL_CUDA(p, cudaGetLastError());
-  if (a.all_segments) FL_CUDA(p, cudaLaunchKernelEx(&cfg, sgmv_expand_kernel<TM, RMAX, true>, a));
-  else FL_CUDA(p, cudaLaunchKernelEx(&cfg, sgmv_expand_kernel<TM, RMAX, false>, a));
+  if (a.all_segments) FL_CUDA(p, launch_pdl(sgmv_expand_kernel<TM, RMAX, true>, egrid, dim3(SG_THREADS), expand_smem, st, a));
+  else FL_CUDA(p, launch_pdl(sgmv_expand_kernel<TM, RMAX, false>, egrid, dim3(SG_THREADS), expand_smem, st, a));
   return FL_OK;
 }
 

@@ -113,4 +113,4 @@ def test_library_tick_on_a_large_tree_is_fast():
     d, order = fl.fl_swapper_decide(arr, prm, used, int(used / 0.97))
     dt = time.perf_counter() - t0
     assert d == -1 and len(order) > 0
-    assert dt < 0.25, dt      # the paper reports under 5 ms for monitoring plus decision; see the design doc for the measured time
+    assert dt < 0.25, dt      # the paper reports under 5 ms for monitoring plus decision; this bound only catches a gross regression

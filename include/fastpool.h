@@ -289,6 +289,16 @@ int fl_swap_eval(const fl_node_stat* nodes, int n, const fl_swap_params* prm, do
 int fl_swapper_decide(const fl_node_stat* nodes, int n, const fl_swap_params* prm, uint32_t blocks_used,
                       uint32_t blocks_total, int32_t* order, int* n_order, int* direction);
 
+/* The ablations of Section 6 ("Effectiveness of the Cache Swapper", "Effectiveness of the Enough LoRAs"): the same
+ * tick with parts of the cost model switched off.  FL_POLICY_LRU: candidates are ordered by last use alone (the
+ * node used longest ago leaves first, the node used last enters first) instead of Eq. 6.  FL_POLICY_NO_LORA_REWARD:
+ * the coefficient of Eq. 4 is 1 for every node.  policy = 0 is fl_swapper_decide.  Unlike fl_swapper_decide,
+ * blocks_used may exceed blocks_total: a caller that needs room for blocks it has not allocated yet adds them to
+ * blocks_used, and the swap-out list then frees enough for usage to fall back to `upper`. */
+enum { FL_POLICY_LRU = 1, FL_POLICY_NO_LORA_REWARD = 2 };
+int fl_swapper_decide_policy(const fl_node_stat* nodes, int n, const fl_swap_params* prm, uint32_t blocks_used,
+                             uint32_t blocks_total, uint32_t policy, int32_t* order, int* n_order, int* direction);
+
 /* ---------------------------------------------------------------- usage dependency tree (Section 4; host code)
  * Virtual root -> LoRA nodes (second layer) -> KV nodes, one per pool block of block_tokens tokens, labelled
  * by those tokens; conversations with a common prefix share its nodes.  The tree only records block ids
@@ -324,6 +334,14 @@ int fl_tree_stats(fl_tree* tree, fl_node_stat* out, int cap, int* n_nodes, doubl
 /* Records a finished swap of `node` with its new block ids.  FL_EBUSY if the move would break the rule of
  * Section 4.2 (a node with a child in HBM may not leave; a node whose parent is in host memory may not enter). */
 int fl_tree_set_location(fl_tree* tree, int32_t node, int in_hbm, const uint32_t* blocks, uint32_t n_blocks);
+/* FL_TREE_OPT_DEPENDENCY (default 1).  0 = the ablation of Section 6 "Effectiveness of the Cache Manager": usage
+ * dependencies are ignored, fl_tree_stats offers every node as a candidate and fl_tree_set_location refuses no
+ * move, so KV nodes can stay in HBM below a node that has left ("invalid KV caches").
+ * fl_tree_invalid counts them: *hbm_kv = KV nodes in HBM, *invalid_kv = those with an ancestor (their adapter
+ * included) outside HBM. */
+enum { FL_TREE_OPT_DEPENDENCY = 0 };
+int fl_tree_set_option(fl_tree* tree, int option, int value);
+int fl_tree_invalid(fl_tree* tree, uint32_t* invalid_kv, uint32_t* hbm_kv);
 /* Verifies that every node in HBM has its parent in HBM ("all KV caches that reside in the HBM are valid").
  * FL_EBADID and *first_bad (may be NULL) on a violation. */
 int fl_tree_check(fl_tree* tree, int32_t* first_bad);

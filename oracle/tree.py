@@ -23,8 +23,11 @@ class TreeError(Exception):
 
 
 class Tree:
-    def __init__(self, bt):
+    def __init__(self, bt, dependency=True):
+        """dependency=False is the paper's ablation "WOM" (Section 6): usage dependencies are ignored, every node is
+        a swap candidate and no move is refused, so KV nodes may stay in HBM below a node that has left."""
         self.bt = bt
+        self.dependency = dependency
         self.nodes = []          # dicts: parent, kind, lora_id, in_hbm, visits, last_use_s, blocks, children {label: id}
         self.lora_node = {}
         self.total_visits = 0.0
@@ -85,7 +88,9 @@ class Tree:
         """Per node: dict for the swapper (candidate flags per Section 4.2), plus total visits and adapters in HBM."""
         out = []
         for i, nd in enumerate(self.nodes):
-            if nd["in_hbm"]:
+            if not self.dependency:
+                cand = True
+            elif nd["in_hbm"]:
                 cand = self._hbm_children(i) == 0
             else:
                 cand = nd["parent"] < 0 or self.nodes[nd["parent"]]["in_hbm"]
@@ -99,12 +104,26 @@ class Tree:
         in_hbm = bool(in_hbm)
         if len(blocks) != len(nd["blocks"]) or in_hbm == nd["in_hbm"]:
             raise TreeError("bad move")
-        if not in_hbm and self._hbm_children(n) != 0:
+        if self.dependency and not in_hbm and self._hbm_children(n) != 0:
             raise TreeError("only a leaf of the HBM part may leave")
-        if in_hbm and nd["parent"] >= 0 and not self.nodes[nd["parent"]]["in_hbm"]:
+        if self.dependency and in_hbm and nd["parent"] >= 0 and not self.nodes[nd["parent"]]["in_hbm"]:
             raise TreeError("only a root of the host part may enter")
         nd["in_hbm"] = in_hbm
         nd["blocks"] = [int(b) for b in blocks]
 
     def valid(self):
         return all(not nd["in_hbm"] or nd["parent"] < 0 or self.nodes[nd["parent"]]["in_hbm"] for nd in self.nodes)
+
+    def invalid(self):
+        """(KV nodes in HBM that some ancestor outside HBM makes unusable, KV nodes in HBM): Section 3's
+        "invalid KV caches"."""
+        bad = total = 0
+        for i, nd in enumerate(self.nodes):
+            if nd["kind"] != KV or not nd["in_hbm"]:
+                continue
+            total += 1
+            p = nd["parent"]
+            while p >= 0 and self.nodes[p]["in_hbm"]:
+                p = self.nodes[p]["parent"]
+            bad += 1 if p >= 0 else 0
+        return bad, total

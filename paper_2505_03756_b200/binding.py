@@ -99,6 +99,10 @@ _SIGS = {
     "fl_tree_stats": (C.c_int, [_vp, C.POINTER(fl_node_stat), C.c_int, C.POINTER(C.c_int), C.POINTER(C.c_double), _i32p]),
     "fl_tree_set_location": (C.c_int, [_vp, C.c_int32, C.c_int, _vp, C.c_uint32]),
     "fl_tree_check": (C.c_int, [_vp, _i32p]),
+    "fl_tree_set_option": (C.c_int, [_vp, C.c_int, C.c_int]),
+    "fl_tree_invalid": (C.c_int, [_vp, _u32p, _u32p]),
+    "fl_swapper_decide_policy": (C.c_int, [C.POINTER(fl_node_stat), C.c_int, C.POINTER(fl_swap_params), C.c_uint32,
+                                           C.c_uint32, C.c_uint32, _vp, C.POINTER(C.c_int), C.POINTER(C.c_int)]),
     "fl_expected_lora_demand": (C.c_int, [_vp, C.c_int, C.c_int, C.POINTER(C.c_double)]),
     "fl_swap_eval": (C.c_int, [C.POINTER(fl_node_stat), C.c_int, C.POINTER(fl_swap_params), _vp]),
     "fl_swapper_decide": (C.c_int, [C.POINTER(fl_node_stat), C.c_int, C.POINTER(fl_swap_params), C.c_uint32, C.c_uint32,
@@ -398,6 +402,20 @@ def fl_swapper_decide(nodes, prm, blocks_used, blocks_total):
     return d.value, order[:n.value].tolist()
 
 
+FL_POLICY_LRU, FL_POLICY_NO_LORA_REWARD = 1, 2
+FL_TREE_OPT_DEPENDENCY = 0
+
+
+def fl_swapper_decide_policy(nodes, prm, blocks_used, blocks_total, policy):
+    """fl_swapper_decide with parts of the cost model switched off (policy flags); blocks_used may exceed the total."""
+    arr = nodes if isinstance(nodes, C.Array) else _nodes(nodes)
+    order = np.empty(max(len(arr), 1), dtype=np.int32)
+    n, d = C.c_int(), C.c_int()
+    _check(lib.fl_swapper_decide_policy(arr, len(arr), C.byref(_params(prm)), blocks_used, blocks_total, policy,
+                                        order.ctypes.data, C.byref(n), C.byref(d)), "fl_swapper_decide_policy")
+    return d.value, order[:n.value].tolist()
+
+
 # ------------------------------------------------------------------ usage dependency tree (host side)
 def fl_tree_create(block_tokens):
     h = _vp()
@@ -468,6 +486,17 @@ def fl_tree_set_location(tree, node, in_hbm, blocks):
 def fl_tree_check(tree):
     bad = C.c_int32(-1)
     return lib.fl_tree_check(tree, C.byref(bad)), bad.value
+
+
+def fl_tree_set_option(tree, option, value):
+    _check(lib.fl_tree_set_option(tree, option, value), "fl_tree_set_option")
+
+
+def fl_tree_invalid(tree):
+    """(KV nodes in HBM with an ancestor outside HBM, KV nodes in HBM)."""
+    bad, total = C.c_uint32(0), C.c_uint32(0)
+    _check(lib.fl_tree_invalid(tree, C.byref(bad), C.byref(total)), "fl_tree_invalid")
+    return int(bad.value), int(total.value)
 
 
 # ------------------------------------------------------------------ views of the two slabs (for tests and tools)

@@ -40,8 +40,14 @@ int fl_swap_eval(const fl_node_stat* nodes, int n, const fl_swap_params* prm, do
 
 int fl_swapper_decide(const fl_node_stat* nodes, int n, const fl_swap_params* prm, uint32_t blocks_used,
                       uint32_t blocks_total, int32_t* order, int* n_order, int* direction) {
-  if (!nodes || !prm || !order || !n_order || !direction || n < 0 || blocks_total == 0 || blocks_used > blocks_total)
-    return FL_EINVAL;
+  if (blocks_used > blocks_total) return FL_EINVAL;
+  return fl_swapper_decide_policy(nodes, n, prm, blocks_used, blocks_total, 0u, order, n_order, direction);
+}
+
+int fl_swapper_decide_policy(const fl_node_stat* nodes, int n, const fl_swap_params* prm, uint32_t blocks_used,
+                             uint32_t blocks_total, uint32_t policy, int32_t* order, int* n_order, int* direction) {
+  if (!nodes || !prm || !order || !n_order || !direction || n < 0 || blocks_total == 0) return FL_EINVAL;
+  if (policy & ~(uint32_t)(FL_POLICY_LRU | FL_POLICY_NO_LORA_REWARD)) return FL_EINVAL;
   if (!(prm->lower >= 0.0 && prm->lower <= prm->upper && prm->upper <= 1.0)) return FL_EINVAL;
   *n_order = 0;
   *direction = 0;
@@ -49,8 +55,15 @@ int fl_swapper_decide(const fl_node_stat* nodes, int n, const fl_swap_params* pr
   const bool out = usage > prm->upper, in = usage < prm->lower;
   if (!out && !in) return FL_OK;                       // between the thresholds: nothing moves
   std::vector<double> eval((size_t)n);
-  int rc = fl_swap_eval(nodes, n, prm, eval.data());
-  if (rc != FL_OK) return rc;
+  if (policy & FL_POLICY_LRU) {
+    // the ablation without the cost model: the node used longest ago leaves first, the one used last enters first
+    for (int i = 0; i < n; ++i) eval[i] = nodes[i].last_use_s;
+  } else {
+    fl_swap_params q = *prm;
+    if (policy & FL_POLICY_NO_LORA_REWARD) q.low_lora = 0.0;     // Eq. 4 coefficient = 1 for every node
+    int rc = fl_swap_eval(nodes, n, &q, eval.data());
+    if (rc != FL_OK) return rc;
+  }
   std::vector<int32_t> cand;
   for (int i = 0; i < n; ++i)
     if (nodes[i].candidate && (nodes[i].in_hbm != 0) == out) cand.push_back(i);

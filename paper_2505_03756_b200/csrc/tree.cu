@@ -40,6 +40,7 @@ uint64_t label_hash(const int32_t* tok, int n) {
 
 struct fl_tree {
   int bt = 16;
+  bool dependency = true;   // false: the ablation that ignores usage dependencies (any node may move)
   std::vector<Node> nodes;
   std::unordered_map<int32_t, int32_t> lora_node;   // lora id -> node
   double total_visits = 0.0;
@@ -173,7 +174,7 @@ int fl_tree_stats(fl_tree* t, fl_node_stat* out, int cap, int* n_nodes, double* 
     out[i].kind = nd.kind;
     out[i].in_hbm = nd.in_hbm;
     // swap-out candidates: HBM nodes with no child in HBM; swap-in candidates: host nodes right below HBM (or the root)
-    out[i].candidate = nd.in_hbm ? (nd.hbm_children == 0) : (nd.parent < 0 || t->nodes[nd.parent].in_hbm);
+    out[i].candidate = !t->dependency ? 1 : nd.in_hbm ? (nd.hbm_children == 0) : (nd.parent < 0 || t->nodes[nd.parent].in_hbm);
     out[i].n_blocks = (uint32_t)nd.blocks.size();
     out[i].visits = nd.visits;
     out[i].last_use_s = nd.last_use_s;
@@ -187,11 +188,38 @@ int fl_tree_set_location(fl_tree* t, int32_t node, int in_hbm, const uint32_t* b
   in_hbm = in_hbm ? 1 : 0;
   if (n_blocks != nd.blocks.size()) return FL_EINVAL;
   if (in_hbm == nd.in_hbm) return FL_EINVAL;
-  if (!in_hbm && nd.hbm_children != 0) return FL_EBUSY;                               // only leaves of the HBM part leave
-  if (in_hbm && nd.parent >= 0 && !t->nodes[nd.parent].in_hbm) return FL_EBUSY;       // only roots of the host part enter
+  if (t->dependency) {
+    if (!in_hbm && nd.hbm_children != 0) return FL_EBUSY;                             // only leaves of the HBM part leave
+    if (in_hbm && nd.parent >= 0 && !t->nodes[nd.parent].in_hbm) return FL_EBUSY;     // only roots of the host part enter
+  }
   nd.in_hbm = in_hbm;
   nd.blocks.assign(blocks, blocks + n_blocks);
   if (nd.parent >= 0) t->nodes[nd.parent].hbm_children += in_hbm ? 1 : -1;
+  return FL_OK;
+}
+
+int fl_tree_set_option(fl_tree* t, int option, int value) {
+  if (!t) return FL_EINVAL;
+  if (option != FL_TREE_OPT_DEPENDENCY) return FL_EINVAL;
+  t->dependency = value != 0;
+  return FL_OK;
+}
+
+int fl_tree_invalid(fl_tree* t, uint32_t* invalid_kv, uint32_t* hbm_kv) {
+  if (!t || !invalid_kv || !hbm_kv) return FL_EINVAL;
+  // nodes are created parents first, so one pass in id order knows every ancestor's state
+  std::vector<char> usable(t->nodes.size());
+  uint32_t bad = 0, all = 0;
+  for (size_t i = 0; i < t->nodes.size(); ++i) {
+    const Node& nd = t->nodes[i];
+    usable[i] = nd.in_hbm && (nd.parent < 0 || usable[nd.parent]);
+    if (nd.kind == FL_NODE_KV && nd.in_hbm) {
+      ++all;
+      bad += usable[i] ? 0u : 1u;
+    }
+  }
+  *invalid_kv = bad;
+  *hbm_kv = all;
   return FL_OK;
 }
 

@@ -350,3 +350,36 @@ def make_workload(name: str, *, n_req: Optional[int] = None, len_range: Optional
     return Workload(name=name, seed=seed, shape=shp, ranks=ranks, scale=2.0, lora_of_req=lora,
                     prefix_lens=prefix, new_lens=new, pool_blocks=pool_blocks,
                     host_blocks=0, popularity=pop)
+
+
+# ---------------------------------------------------------------------------------------------------------------
+# Multi-turn conversation traces for the cache manager / swapper (no arithmetic of the method here).
+def conversation_trace(seed: int, n_lora: int, n_conv: int, n_turns: int, popularity: str = "uniform",
+                       block_tokens: int = 16, system_blocks: int = 2, turn_tokens=(8, 72)):
+    """Events (lora_id, tokens) of multi-turn chats: every turn repeats its conversation so far and adds new
+    tokens; all conversations of an adapter start with that adapter's system prompt.  How conversations pick
+    their adapter follows the paper's large-LoRA-count study (Section 6): "uniform" (equal probability),
+    "distinct" (adapters taken in turn) or "skewed-x" (a Gaussian over the adapter index with standard
+    deviation x, centred on the middle adapter)."""
+    rs = Stream(seed, "conversation-trace/" + popularity)
+    if popularity == "uniform":
+        owner = rs.integers(0, n_lora - 1, n_conv)
+    elif popularity == "distinct":
+        owner = np.arange(n_conv, dtype=np.int64) % n_lora
+    elif popularity.startswith("skewed-"):
+        std = float(popularity.split("-", 1)[1])
+        owner = np.clip(np.rint(n_lora / 2 + rs.normal((n_conv,), std)), 0, n_lora - 1).astype(np.int64)
+    else:
+        raise ValueError(popularity)
+    system = {a: [int(v) for v in rs.integers(1, 999, system_blocks * block_tokens)] for a in range(n_lora)}
+    convs = [dict(lora=int(owner[c]), tokens=[]) for c in range(n_conv)]
+    events = []
+    for _ in range(n_turns):
+        for ci in rs.permutation(n_conv):
+            c = convs[int(ci)]
+            if not c["tokens"]:
+                c["tokens"] = list(system[c["lora"]])
+            n_new = int(rs.integers(turn_tokens[0], turn_tokens[1], 1)[0])
+            c["tokens"] = c["tokens"] + [int(v) for v in rs.integers(1000, 30000, n_new)]
+            events.append((c["lora"], list(c["tokens"])))
+    return events

@@ -705,6 +705,14 @@ int sgmv_common(fl_pool* p, fl_bf16* const* ys, const fl_bf16* x, const int* mat
   const bool small = n_tokens <= 16 * n_seg;   // average segment of at most 16 tokens: decode-like
   const int rmax = rmax_of(p);
   const cudaStream_t st = (cudaStream_t)stream;
+  if (!small && rmax == 16 && a.ksplit == 1) {
+    // A long-segment batch of a few thousand tokens gives the shrink about two CTAs per SM (eight warps), too few to
+    // keep the loads of a rank-16 shrink in flight: two slices of d_in double them.  The scratch is sized for rank 64,
+    // so at rank 16 two slices fit in what the caller already brought.
+    const long shrink_ctas = (long)(n_seg + n_tokens / 64) * (n_mats == 3 ? 1 : n_mats);
+    const size_t need = (size_t)n_mats * 2 * (size_t)n_tokens * rmax * sizeof(float) + 256;
+    if (shrink_ctas < 592 && need <= workspace_bytes) a.ksplit = 2;
+  }
   int rc;
   if (small) {
     const int tiles = n_seg + n_tokens / 16;

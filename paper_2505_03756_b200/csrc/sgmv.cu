@@ -19,7 +19,7 @@ constexpr int SG_THREADS = 128;
 constexpr int KS = 64;            // d_in elements per shrink pipeline stage (128-byte rows)
 constexpr int SH_STAGES = 4;
 constexpr int NSUB = 128;         // y columns per expand sub-tile (256-byte rows)
-constexpr int EXPAND_COLS_MIN = 512, EXPAND_COLS_MAX = 4096;   // y columns per expand CTA: picked per call
+constexpr int EXPAND_COLS_MIN = 512, EXPAND_COLS_MAX = 2048;   // y columns per expand CTA: picked per call
 constexpr int KSPLIT_MAX = 8;
 
 struct SgmvArgs {

@@ -440,7 +440,7 @@ int launch_prefill_tc2(fl_pool* p, const AttnArgs& a, int n_tokens, int max_item
   }
   const int group = a.n_q / a.n_kv;
   const int heads_per_item = group % 2 == 0 ? a.n_q / 2 : a.n_q;
-  // one CTA per SM (shared memory and TMEM allow no more); CTAs beyond the plan's unit count exit at once
+  // one CTA per SM (shared memory and TMEM allow no more); a CTA beyond the plan's unit count finds no work and tears down
   const long long units = (long long)max_items * heads_per_item;
   const unsigned grid = (unsigned)std::min<long long>(units, p->sm_count);
   if (grid == 0) return FL_OK;

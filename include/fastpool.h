@@ -63,6 +63,8 @@ typedef struct {
   uint32_t blocks_used, blocks_free, host_blocks_used, host_blocks_free;
   uint32_t lora_blocks;         /* device blocks referenced by registered adapters */
   uint64_t bytes_swapped_in, bytes_swapped_out;
+  uint64_t staging_bytes;       /* device memory the pool holds outside the slab for the swap path's two staging
+                                   areas (see fl_swap_out); 0 when the pool has fewer than two host blocks */
 } fl_status;
 
 /* ---------------------------------------------------------------- pool (Section 4.3)
@@ -98,11 +100,16 @@ int fl_pool_snapshot(fl_pool* pool, int host, uint32_t* free_ids, uint32_t cap, 
 /* Reads the sticky device flags (synchronises the device) and the counters.  clear != 0 resets the flags. */
 int fl_pool_status(fl_pool* pool, fl_status* out, int clear);
 int fl_last_cuda_error(fl_pool* pool);
-/* Tuning switches.  FL_OPT_PREFILL_KERNEL: 0 (default) = prefill attention on tcgen05 tensor cores with
+/* Switches.  FL_OPT_PREFILL_KERNEL: 0 (default) = prefill attention on tcgen05 tensor cores with
  * TMEM accumulators and TMA-staged pages, two query tiles per CTA sharing the K/V stream; 1 = the
- * mma.sync kernel; 2 = the tcgen05 kernel with one query tile per CTA.  Same results within rounding.
- * The tcgen05 kernels need sm_scale > 0; other values are served by the mma.sync kernel. */
+ * mma.sync kernel.  Same results within rounding.  The tcgen05 kernel needs sm_scale > 0; other values are
+ * served by the mma.sync kernel.
+ * FL_OPT_POISON_FREED: 1 = debugging aid that stands in for a memory checker: fl_block_free waits for the
+ * device and fills every freed DEVICE block with 0xFF bytes (bf16 NaN patterns), so a block table that still
+ * names a freed block turns the output of whatever reads it into NaN instead of plausible numbers.  0 (default)
+ * = freed blocks keep their contents and fl_block_free touches no device memory. */
 #define FL_OPT_PREFILL_KERNEL 1
+#define FL_OPT_POISON_FREED 2
 int fl_pool_set_option(fl_pool* pool, int key, int value);
 
 /* ---------------------------------------------------------------- adapters (Section 4.3)
@@ -130,6 +137,30 @@ int fl_lora_pack_host(fl_pool* pool, int32_t rank, const fl_lora_shape* mats, in
 int fl_lora_register(fl_pool* pool, int32_t lora_id, int32_t rank, const fl_lora_shape* mats, int n_mats,
                      const uint32_t* block_table, uint32_t n_table);
 int fl_lora_unregister(fl_pool* pool, int32_t lora_id);
+/* Both calls wait for the device before they change the directory (kernels of any stream may be reading it).
+ * A CUDA graph recorded from the compute calls keeps the directory's address and the rank its kernels were
+ * built for: record it again after a registration that raises the pool's highest rank past 16 or 32, or whose
+ * id is 4096 or more above every id registered before (the directory grows by doubling).  A kernel that meets
+ * an adapter of a higher rank than it was built for leaves out the extra rank-rows and sets bit 2 of
+ * device_flags. */
+
+/* Read-back of what the DEVICE holds for adapter `lora_id` (Section 4.3: block tables record where each block
+ * is): its directory entry and its block table, copied from device memory.  For every projection m: class table
+ * entry, first row inside the class and rows per block of the A rows (a_*) and of the B rows (b_*), as defined
+ * above.  table (host pointer, capacity cap; may be NULL) receives the n_table block ids, *n_table (may be
+ * NULL) their count; table_off is the adapter's first entry inside the pool's table arena.  Synchronises the
+ * device.  FL_EBADID: no such adapter. */
+typedef struct {
+  uint32_t a_tab, a_row0, a_rpb, b_tab, b_row0, b_rpb;
+  int32_t d_in, d_out;
+} fl_lora_mat_placement;
+typedef struct {
+  int32_t rank, n_mats;
+  uint32_t table_off, n_table;
+  fl_lora_mat_placement mats[FL_MAX_MATS];
+} fl_lora_placement;
+int fl_lora_snapshot(fl_pool* pool, int32_t lora_id, fl_lora_placement* out, uint32_t* table, uint32_t cap,
+                     uint32_t* n_table);
 
 /* ---------------------------------------------------------------- LoRA projection (Eq. 1, Eq. 2; Section 2.1 SGMV)
  * For every segment s (tokens seg_indptr[s] .. seg_indptr[s+1]) with adapter i = lora_ids[s]:
@@ -158,6 +189,7 @@ int fl_lora_sgmv_multi(fl_pool* pool, fl_bf16* const* ys, const fl_bf16* x, cons
  * Segments with lora_ids[s] < 0 get their base k, v copied into the pool.  mat_k and mat_v must have
  * d_out = n_kv_heads * 128 and the three projections share x; req_indptr .. prefix_lens as in fl_kv_append;
  * workspace as in fl_lora_sgmv_multi with n_mats = 3. */
+/* Blocks of up to 128 tokens and pools of up to 2^24 blocks (FL_EINVAL beyond). */
 int fl_lora_sgmv_qkv_append(fl_pool* pool, fl_bf16* y_q, const fl_bf16* y_k, const fl_bf16* y_v, const fl_bf16* x,
                             int mat_q, int mat_k, int mat_v, const int32_t* seg_indptr, const int32_t* lora_ids,
                             int n_seg, int n_tokens, float scale, const int32_t* req_indptr,
@@ -178,7 +210,8 @@ int fl_lora_sgmv_qkv_append(fl_pool* pool, fl_bf16* y_q, const fl_bf16* y_k, con
  *    FL_SGMV_STATIC_BYTES; the 8 MiB cover every batch of up to 32767 tokens.
  *  - The first call on a device looks up the array's device address (one runtime query, remembered
  *    per device); make that first call outside any stream capture.
- *  - All calls on one device share the array, and it keeps whatever the last call left in it.  The
+ *  - All calls on one device, from every pool and every thread of the process, share the array (its address
+ *    is remembered per process, not per pool), and it keeps whatever the last call left in it.  The
  *    kernels overwrite every value they later read, so nothing has to be cleared between calls, but two
  *    calls whose kernels may overlap on the GPU (different streams without an ordering between them)
  *    race on it: keep such calls on one stream or order them with events. */
@@ -222,9 +255,11 @@ int fl_paged_attention(fl_pool* pool, fl_bf16* out, const fl_bf16* q, const int3
  * streams.  Every listed block must be allocated (FL_EBADID) and no block may be listed twice in one
  * call (FL_EINVAL); on either error nothing is copied.  The transfers run on the copy engines: pairs
  * that are consecutive in both memories go as one DMA; a run of consecutive host blocks whose device
- * blocks are scattered goes through a staging area inside the pool (one small gather or scatter kernel
- * on `side` plus one DMA for up to 256 blocks), which is what a fragmented pool needs to keep the host
- * link busy.  Swap-out and swap-in have separate staging areas, so the two directions overlap when they
+ * blocks are scattered goes through a staging area (one small gather or scatter kernel on `side` plus one
+ * DMA for up to 256 blocks), which is what a fragmented pool needs to keep the host link busy.  The two
+ * staging areas are device memory that fl_pool_create allocates OUTSIDE the slab: min(256, n_blocks,
+ * n_host_blocks) blocks each (128 MiB in all at 256 KiB blocks), none when the pool has fewer than two host
+ * blocks; fl_pool_status reports the total as staging_bytes.  Swap-out and swap-in have separate staging areas, so the two directions overlap when they
  * are given different streams; calls in one direction are ordered among themselves by the library even
  * across streams.  The caller guarantees that no kernel in flight touches the listed device blocks
  * (the paper evicts only nodes no running query uses, and a query whose blocks are in flight waits).

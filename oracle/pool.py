@@ -22,7 +22,8 @@ used; allocator replayed against brute-force set bookkeeping (no id handed out t
 = n_blocks, a failed call changes nothing, LIFO order on a hand-written trace); swap-out followed
 by swap-in elsewhere returns identical bytes and touches no other block; adapter block counts for
 the paper-shaped layers (2 blocks for a 7B rank-8 adapter, 16 for the 13B rank-32 adapter with MLP,
-100 for the 34B rank-64 adapter).
+100 for the 34B rank-64 adapter); table entry and byte offset of single adapter elements of the 34B
+rank-64 adapter worked out by hand (both width classes, first and last value of a block).
 """
 import numpy as np
 

@@ -46,7 +46,17 @@ class fl_swap_params(C.Structure):
 class fl_status(C.Structure):
     _fields_ = [("device_flags", C.c_uint32), ("blocks_used", C.c_uint32), ("blocks_free", C.c_uint32),
                 ("host_blocks_used", C.c_uint32), ("host_blocks_free", C.c_uint32), ("lora_blocks", C.c_uint32),
-                ("bytes_swapped_in", C.c_uint64), ("bytes_swapped_out", C.c_uint64)]
+                ("bytes_swapped_in", C.c_uint64), ("bytes_swapped_out", C.c_uint64), ("staging_bytes", C.c_uint64)]
+
+
+class fl_lora_mat_placement(C.Structure):
+    _fields_ = [("a_tab", C.c_uint32), ("a_row0", C.c_uint32), ("a_rpb", C.c_uint32), ("b_tab", C.c_uint32),
+                ("b_row0", C.c_uint32), ("b_rpb", C.c_uint32), ("d_in", C.c_int32), ("d_out", C.c_int32)]
+
+
+class fl_lora_placement(C.Structure):
+    _fields_ = [("rank", C.c_int32), ("n_mats", C.c_int32), ("table_off", C.c_uint32), ("n_table", C.c_uint32),
+                ("mats", fl_lora_mat_placement * 8)]
 
 
 _vp, _u32p, _i32p = C.c_void_p, C.POINTER(C.c_uint32), C.POINTER(C.c_int32)
@@ -70,6 +80,7 @@ _SIGS = {
                                     C.POINTER(_vp), _vp, C.c_uint32]),
     "fl_lora_register": (C.c_int, [_vp, C.c_int32, C.c_int32, C.POINTER(fl_lora_shape), C.c_int, _vp, C.c_uint32]),
     "fl_lora_unregister": (C.c_int, [_vp, C.c_int32]),
+    "fl_lora_snapshot": (C.c_int, [_vp, C.c_int32, C.POINTER(fl_lora_placement), _vp, C.c_uint32, _u32p]),
     "fl_lora_sgmv_workspace": (C.c_size_t, [C.c_int, C.c_int]),
     "fl_lora_sgmv": (C.c_int, [_vp, _vp, _vp, C.c_int, _vp, _vp, C.c_int, C.c_int, C.c_float, _vp, C.c_size_t, _vp]),
     "fl_lora_sgmv_static": (C.c_int, [_vp, _vp, _vp, C.c_int, _vp, _vp, C.c_int, C.c_int, C.c_float, _vp]),
@@ -221,6 +232,7 @@ def fl_last_cuda_error(pool):
 
 
 FL_OPT_PREFILL_KERNEL = 1
+FL_OPT_POISON_FREED = 2
 
 
 def fl_pool_set_option(pool, key, value):
@@ -250,6 +262,17 @@ def fl_lora_register(pool, lora_id, rank, mats, block_table):
 
 def fl_lora_unregister(pool, lora_id):
     _check(lib.fl_lora_unregister(pool, lora_id), "fl_lora_unregister")
+
+
+def fl_lora_snapshot(pool, lora_id):
+    """What the device holds for the adapter: ({rank, n_mats, table_off, n_table, mats: [dict per projection]}, block table)."""
+    pl = fl_lora_placement()
+    n = C.c_uint32()
+    _check(lib.fl_lora_snapshot(pool, lora_id, C.byref(pl), None, 0, C.byref(n)), "fl_lora_snapshot")
+    table = np.empty(n.value, dtype=np.uint32)
+    _check(lib.fl_lora_snapshot(pool, lora_id, C.byref(pl), table.ctypes.data, n.value, C.byref(n)), "fl_lora_snapshot")
+    mats = [{k: getattr(pl.mats[m], k) for k, _ in fl_lora_mat_placement._fields_} for m in range(pl.n_mats)]
+    return dict(rank=pl.rank, n_mats=pl.n_mats, table_off=pl.table_off, n_table=pl.n_table, mats=mats), table
 
 
 def fl_lora_sgmv_workspace(n_tokens, n_mats=1):

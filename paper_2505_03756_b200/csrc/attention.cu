@@ -61,7 +61,10 @@ __global__ void __launch_bounds__(256) attn_plan_kernel(const AttnArgs a, int ch
     const int off_p = base_p + block_excl_scan(tiles, sh, tot_p);
     const int off_d = base_d + block_excl_scan(chunks, sh, tot_d);
     if (i < a.n_req) {
-      a.req_info[i] = make_int4(off_d, chunks, dec ? 1 : 0, 0);
+      // a request whose chunks do not all fit in the list (contexts longer than the caller's n_tbl covers) gets no
+      // output: the chunks that did fit only write partial slots inside the workspace, and the merge, which would
+      // read all of them, skips the request (the overflow raises FLAG_BAD_POS below)
+      a.req_info[i] = make_int4(off_d, off_d + chunks > a.max_decode ? 0 : chunks, dec ? 1 : 0, 0);
       for (int t = 0; t < tiles; ++t)
         if (off_p + t < a.max_prefill) a.prefill_tmp[off_p + t] = make_int2(i, t * qt);
       for (int c = 0; c < chunks; ++c)
@@ -557,7 +560,7 @@ int fl_paged_attention(fl_pool* p, fl_bf16* out, const fl_bf16* q, const int32_t
     // every kernel of the call is a programmatic dependent launch: it may start while the one before it drains
     // and waits inside for that kernel's results
     if (launch_pdl(attn_plan_kernel, dim3(1), dim3(256), 0, st, a, w.chunk,
-                   kind == 0 ? tc2_tile_tokens(n_q_heads, n_kv_heads) : (kind == 2 ? QT_TC : QT_MMA)) != cudaSuccess) {
+                   kind == 0 ? tc2_tile_tokens(n_q_heads, n_kv_heads) : QT_MMA) != cudaSuccess) {
       p->last_cuda = (int)cudaGetLastError();
       rc = FL_ECUDA;
       break;
@@ -569,9 +572,6 @@ int fl_paged_attention(fl_pool* p, fl_bf16* out, const fl_bf16* q, const int32_t
       const int max_req = std::min(n_req, n_tokens / (DEC_ROWS / group + 1));
       const int max_items = std::min(w.max_prefill, n_tokens / tc2_tile_tokens(n_q_heads, n_kv_heads) + max_req);
       rc = launch_prefill_tc2(p, a, n_tokens, max_items, st);
-      if (rc != FL_OK) break;
-    } else if (kind == 2) {
-      rc = launch_prefill_tc(p, a, n_tokens, st);
       if (rc != FL_OK) break;
     } else {
       attn_prefill_kernel<<<(unsigned)w.max_prefill * n_q_heads, ATT_THREADS, PRE_SMEM, st>>>(a);

@@ -2,15 +2,12 @@
 #pragma once
 #include "pool.cuh"
 
-struct CUtensorMap_st;
-
 namespace attn {
 
 constexpr int D = FL_HEAD_DIM;
 constexpr int BT = 16;                 // tokens per block these kernels cover
 constexpr int PAGE_BYTES = BT * D * 2;   // one (block, kv head, K or V) piece
 constexpr int QT_MMA = 64;             // query rows per prefill tile, mma.sync kernel
-constexpr int QT_TC = 128;             // query rows per prefill tile, tcgen05 kernel
 constexpr int KT = 64;                 // keys per prefill iteration
 constexpr int ATT_THREADS = 128;
 constexpr int DEC_ROWS = 16;
@@ -43,10 +40,6 @@ struct AttnArgs {
 };
 
 
-// Tensor maps of the pool slab (cached in the pool) and of q, as the tcgen05 prefill kernels read them.
-int prefill_tensor_maps(fl_pool* p, const AttnArgs& a, int n_tokens, const ::CUtensorMap_st** kv_out, ::CUtensorMap_st* qmap);
-// Launches the one-tile-per-CTA tcgen05/TMEM prefill kernel over the plan's prefill list (tiles of QT_TC rows).
-int launch_prefill_tc(fl_pool* p, const AttnArgs& a, int n_tokens, cudaStream_t st);
 // Launches the two-tiles-per-CTA kernel; the plan's tiles are tc2_tile_tokens(n_q, n_kv) tokens long.
 int launch_prefill_tc2(fl_pool* p, const AttnArgs& a, int n_tokens, int max_items, cudaStream_t st);
 inline int tc2_tile_tokens(int n_q, int n_kv) { return (n_q / n_kv) % 2 == 0 ? 128 : 256; }

@@ -26,6 +26,7 @@
 #include "attention.cuh"
 #include "mma_utils.cuh"
 #include "tc_ptx.cuh"
+#include "tmap.cuh"
 
 namespace attn {
 namespace {
@@ -431,8 +432,15 @@ attn_prefill_tc2_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap kv
 int launch_prefill_tc2(fl_pool* p, const AttnArgs& a, int n_tokens, int max_items, cudaStream_t st) {
   const CUtensorMap* kv = nullptr;
   alignas(64) CUtensorMap qmap;
-  int rc = prefill_tensor_maps(p, a, n_tokens, &kv, &qmap);
+  int rc = tmap::kv_pages(p, a.n_kv, &kv);
   if (rc != FL_OK) return rc;
+  {   // q as [token][head][128]: box = 64 elements x 128 tokens of one head
+    const uint64_t dims[3] = {(uint64_t)D, (uint64_t)a.n_q, (uint64_t)n_tokens};
+    const uint64_t strides[2] = {(uint64_t)D * 2, (uint64_t)a.n_q * D * 2};
+    const uint32_t box[3] = {64, 1, 128};
+    rc = tmap::encode_bf16(&qmap, a.q, 3, dims, strides, box);
+    if (rc != FL_OK) return rc;
+  }
   static bool configured[16] = {};
   if (!configured[p->device & 15]) {
     FL_CUDA(p, cudaFuncSetAttribute(attn_prefill_tc2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)T2_SMEM));

@@ -173,7 +173,16 @@ int fl_block_alloc(fl_pool* p, uint32_t n, uint32_t* ids) {
 }
 int fl_block_free(fl_pool* p, uint32_t n, const uint32_t* ids) {
   if (!p || (n && !ids)) return FL_EINVAL;
-  return stack_free(p->dev, n, ids);
+  const int rc = stack_free(p->dev, n, ids);
+  if (rc == FL_OK && p->poison_freed) {
+    // debugging aid: a freed block is filled with bf16 NaN patterns (0xFFFF), behind everything already enqueued
+    // on the device, so that a table that still names it shows up as NaN in whatever reads it
+    DeviceGuard g(p->device);
+    FL_CUDA(p, cudaDeviceSynchronize());
+    for (uint32_t i = 0; i < n; ++i)
+      FL_CUDA(p, cudaMemset(p->slab + (size_t)ids[i] * p->block_bytes, 0xFF, p->block_bytes));
+  }
+  return rc;
 }
 int fl_host_block_alloc(fl_pool* p, uint32_t n, uint32_t* ids) {
   if (!p || (n && !ids)) return FL_EINVAL;
@@ -229,6 +238,7 @@ int fl_pool_status(fl_pool* p, fl_status* out, int clear) {
   out->lora_blocks = p->lora_blocks;
   out->bytes_swapped_in = p->bytes_in;
   out->bytes_swapped_out = p->bytes_out;
+  out->staging_bytes = (uint64_t)2 * p->stage_blocks * p->block_bytes;
   return FL_OK;
 }
 
@@ -236,8 +246,12 @@ int fl_last_cuda_error(fl_pool* p) { return p ? p->last_cuda : 0; }
 
 int fl_pool_set_option(fl_pool* p, int key, int value) {
   if (!p) return FL_EINVAL;
-  if (key == FL_OPT_PREFILL_KERNEL && value >= 0 && value <= 2) {
+  if (key == FL_OPT_PREFILL_KERNEL && value >= 0 && value <= 1) {
     p->prefill_kernel = value;
+    return FL_OK;
+  }
+  if (key == FL_OPT_POISON_FREED && (value == 0 || value == 1)) {
+    p->poison_freed = value;
     return FL_OK;
   }
   return FL_EINVAL;
@@ -277,11 +291,39 @@ int fl_lora_pack_host(fl_pool* p, int32_t rank, const fl_lora_shape* mats, int n
   return FL_OK;
 }
 
+int fl_lora_snapshot(fl_pool* p, int32_t lora_id, fl_lora_placement* out, uint32_t* table, uint32_t cap, uint32_t* n_table) {
+  if (!p || !out || lora_id < 0) return FL_EINVAL;
+  if ((uint32_t)lora_id >= p->dir_cap) return FL_EBADID;
+  DeviceGuard g(p->device);
+  LoraEntry e;
+  FL_CUDA(p, cudaDeviceSynchronize());
+  FL_CUDA(p, cudaMemcpy(&e, p->d_dir + lora_id, sizeof(e), cudaMemcpyDeviceToHost));
+  if (e.rank <= 0) return FL_EBADID;
+  if (e.n_mats < 0 || e.n_mats > FL_MAX_MATS || (size_t)e.table_off + e.n_table > p->tables_cap) return FL_EINVAL;
+  out->rank = e.rank;
+  out->n_mats = e.n_mats;
+  out->table_off = e.table_off;
+  out->n_table = e.n_table;
+  for (int m = 0; m < FL_MAX_MATS; ++m) {
+    const LoraMat& lm = e.mats[m];
+    out->mats[m] = fl_lora_mat_placement{lm.a_tab, lm.a_row0, lm.a_rpb, lm.b_tab, lm.b_row0, lm.b_rpb, lm.d_in, lm.d_out};
+  }
+  if (n_table) *n_table = e.n_table;
+  if (table) {
+    if (cap < e.n_table) return FL_EINVAL;
+    if (e.n_table)
+      FL_CUDA(p, cudaMemcpy(table, p->d_tables + e.table_off, sizeof(uint32_t) * e.n_table, cudaMemcpyDeviceToHost));
+  }
+  return FL_OK;
+}
+
 int fl_lora_unregister(fl_pool* p, int32_t lora_id) {
   if (!p) return FL_EINVAL;
   auto it = p->registered.find(lora_id);
   if (it == p->registered.end()) return FL_EBADID;
   DeviceGuard g(p->device);
+  // kernels on any stream may still be reading the entry and its table range, which is reused right away
+  FL_CUDA(p, cudaDeviceSynchronize());
   FL_CUDA(p, cudaMemset(p->d_dir + lora_id, 0, sizeof(LoraEntry)));
   arena_give(p, it->second.table_off, it->second.n_table);
   p->lora_blocks -= it->second.n_table;
@@ -306,6 +348,7 @@ int fl_lora_register(fl_pool* p, int32_t lora_id, int32_t rank, const fl_lora_sh
   for (uint32_t i = 0; i < n_table; ++i)
     if (block_table[i] >= p->n_blocks || !p->dev.used[block_table[i]]) return FL_EBADID;
   DeviceGuard g(p->device);
+  FL_CUDA(p, cudaDeviceSynchronize());   // no kernel may be reading the directory while it changes
   if (p->registered.count(lora_id)) {
     rc = fl_lora_unregister(p, lora_id);
     if (rc != FL_OK) return rc;
@@ -314,7 +357,6 @@ int fl_lora_register(fl_pool* p, int32_t lora_id, int32_t rank, const fl_lora_sh
     uint32_t cap = p->dir_cap;
     while (cap <= (uint32_t)lora_id) cap *= 2;
     LoraEntry* nd = nullptr;
-    FL_CUDA(p, cudaDeviceSynchronize());
     FL_CUDA(p, cudaMalloc(&nd, sizeof(LoraEntry) * cap));
     FL_CUDA(p, cudaMemset(nd, 0, sizeof(LoraEntry) * cap));
     FL_CUDA(p, cudaMemcpy(nd, p->d_dir, sizeof(LoraEntry) * p->dir_cap, cudaMemcpyDeviceToDevice));

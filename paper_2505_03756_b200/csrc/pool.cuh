@@ -67,7 +67,8 @@ struct fl_pool {
   uint64_t bytes_in = 0, bytes_out = 0;
   int last_cuda = 0;
   int sm_count = 148;
-  int prefill_kernel = 0;                           // 0: tcgen05 two-tile kernel, 1: mma.sync kernel, 2: tcgen05 one-tile kernel
+  int prefill_kernel = 0;                           // 0: tcgen05 two-tile kernel, 1: mma.sync kernel
+  int poison_freed = 0;                             // debugging aid: freed device blocks are filled with NaN patterns
   unsigned char* stage[2] = {nullptr, nullptr};     // contiguous staging areas of the swap path (out, in)
   uint32_t stage_blocks = 0;
   cudaEvent_t stage_done[2] = {nullptr, nullptr};   // last use of each staging area

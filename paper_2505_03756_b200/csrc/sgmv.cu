@@ -129,6 +129,9 @@ __global__ void __launch_bounds__(SG_THREADS) sgmv_shrink_kernel(const SgmvArgs 
   const LoraEntry* e = a.pv.dir + lid;
   const LoraMat lm = e->mats[a.mat_index[j]];
   const int rank = min(e->rank, RMAX);
+  // an adapter of a higher rank than this instantiation covers (registered after the launch was recorded
+  // into a graph): its extra rank-rows are left out, and the status word says so
+  if (e->rank > RMAX && tid == 0) atomicOr(a.pv.flags, (uint32_t)FLAG_BAD_LORA);
   const uint32_t table_off = e->table_off;
   const int d_in = lm.d_in;
   const int kchunk = ((d_in + a.ksplit * KS - 1) / (a.ksplit * KS)) * KS;
@@ -258,6 +261,9 @@ __global__ void __launch_bounds__(SG_THREADS) sgmv_shrink3_kernel(const SgmvArgs
     }
   }
   const int rank = min(e->rank, RMAX);
+  // an adapter of a higher rank than this instantiation covers (registered after the launch was recorded
+  // into a graph): its extra rank-rows are left out, and the status word says so
+  if (e->rank > RMAX && tid == 0) atomicOr(a.pv.flags, (uint32_t)FLAG_BAD_LORA);
   const uint32_t table_off = e->table_off;
   const int d_in = e->mats[a.mat_index[0]].d_in;
   const int kchunk = ((d_in + a.ksplit * KS - 1) / (a.ksplit * KS)) * KS;
@@ -411,7 +417,7 @@ __global__ void __launch_bounds__(SG_THREADS, expand_min_ctas(TM, RMAX, KV)) sgm
   }
   // K / V rows: where each of this thread's token rows lives in the pool (block and slot of its position),
   // and how many slots behind it have to be cleared (V of a request's last token)
-  uint32_t kvloc[KV ? YR : 1];      // block << 5 | slot << 1 | "last token of its request"
+  uint32_t kvloc[KV ? YR : 1];      // block << 8 | slot << 1 | "last token of its request" (slot < 128, block < 2^24)
   if (KV && side >= 0) {
     int r = 0;
     {
@@ -431,18 +437,18 @@ __global__ void __launch_bounds__(SG_THREADS, expand_min_ctas(TM, RMAX, KV)) sgm
       while (r + 1 < a.n_req && t >= a.req_indptr[r + 1]) ++r;
       const int pos = a.prefix_lens[r] + (t - a.req_indptr[r]);
       const int entry = pos / a.bt, slot = pos - entry * a.bt;
-      if (t < a.req_indptr[r] || t >= a.req_indptr[r + 1] || entry >= a.tbl_indptr[r + 1] - a.tbl_indptr[r]) {
+      if (pos < 0 || t < a.req_indptr[r] || t >= a.req_indptr[r + 1] || entry >= a.tbl_indptr[r + 1] - a.tbl_indptr[r]) {
         atomicOr(a.pv.flags, (uint32_t)FLAG_BAD_POS);
         yok[i] = false;
         continue;
       }
       const uint32_t blk = a.tbl[a.tbl_indptr[r] + entry];
-      if (blk >= a.pv.n_blocks || blk >= (1u << 27)) {
+      if (blk >= a.pv.n_blocks || blk >= (1u << 24)) {
         atomicOr(a.pv.flags, (uint32_t)FLAG_BAD_BLOCK);
         yok[i] = false;
         continue;
       }
-      kvloc[i] = blk << 5 | (uint32_t)slot << 1 | (t == a.req_indptr[r + 1] - 1 ? 1u : 0u);
+      kvloc[i] = blk << 8 | (uint32_t)slot << 1 | (t == a.req_indptr[r + 1] - 1 ? 1u : 0u);
     }
   }
   const __nv_bfloat16* brow[BR];
@@ -552,8 +558,8 @@ __global__ void __launch_bounds__(SG_THREADS, expand_min_ctas(TM, RMAX, KV)) sgm
           for (int i = 0; i < YR; ++i) {
             if (yok[i]) {
               const uint32_t loc = kvloc[KV ? i : 0];
-              const int slot = (loc >> 1) & 15;
-              unsigned char* dst = a.pv.slab + (size_t)(loc >> 5) * a.pv.block_bytes + head_off + slot * (FL_HEAD_DIM * 2);
+              const int slot = (loc >> 1) & 127;
+              unsigned char* dst = a.pv.slab + (size_t)(loc >> 8) * a.pv.block_bytes + head_off + slot * (FL_HEAD_DIM * 2);
               *reinterpret_cast<uint4*>(dst) = add_bf16x8(*reinterpret_cast<const uint4*>(ysm + swz(crow + 8 * i, cchunk, 16)),
                                                           *reinterpret_cast<const uint4*>(dsm + swz(crow + 8 * i, cchunk, 16)));
               if (side == 1 && (loc & 1u))     // V of a request's last token: clear the slots behind it
@@ -689,6 +695,8 @@ int sgmv_common(fl_pool* p, fl_bf16* const* ys, const fl_bf16* x, const int* mat
     a.n_req = kv->n_req;
     a.n_kv = kv->n_kv;
     a.bt = (int)(p->block_bytes / per_tok);
+    // the expand packs a token's destination into one word: 7 bits of slot, 24 bits of block id
+    if (a.bt > 128 || p->n_blocks > (1u << 24)) return FL_EINVAL;
   }
   a.n_mats = n_mats;
   a.seg_indptr = seg_indptr;
@@ -769,7 +777,7 @@ static __device__ __align__(256) unsigned char g_sgmv_static_scratch[FL_SGMV_STA
 
 namespace {
 constexpr int STATIC_MAX_DEVICES = 64;
-void* g_static_scratch_addr[STATIC_MAX_DEVICES] = {};   // device address of the array, per device
+void* g_static_scratch_addr[STATIC_MAX_DEVICES] = {};   // device address of the array, per device; one copy per process
 }  // namespace
 
 extern "C" {
@@ -779,6 +787,7 @@ int fl_lora_sgmv_static(fl_pool* p, fl_bf16* y, const fl_bf16* x, int mat_index,
                         float scale, fl_stream stream) {
   if (!p || n_seg < 0 || n_tokens < 0) return FL_EINVAL;
   if (p->device < 0 || p->device >= STATIC_MAX_DEVICES) return FL_EINVAL;
+  if (n_seg == 0 || n_tokens == 0) return FL_OK;      // nothing to do, as in fl_lora_sgmv
   if (fl_lora_sgmv_workspace(n_tokens, 1) > (size_t)FL_SGMV_STATIC_BYTES) return FL_ENOMEM;   // batch too large for the built-in scratch
   void* scratch = g_static_scratch_addr[p->device];
   if (!scratch) {

@@ -1,17 +1,30 @@
 """Shared helpers of the GPU parity tests: tolerance, and the oracle-side mirror of a Session."""
+import os
+
 import numpy as np
 
 from oracle import pool as op
 from paper_2505_03756_b200 import synth
 
-REL = 1e-2   # spec bound: bf16 inputs, fp32 accumulation, bf16 output
+REL = 1e-2      # bound on the error of an output relative to the tensor: bf16 inputs, fp32 accumulation, bf16 output
+SLACK = 2e-2    # element-wise absolute allowance in units of rms(ref), see assert_close
+
+_observed = {}  # what -> largest (|d| - REL |ref|) / rms(ref) seen, written out when FL_TOL_REPORT names a file
 
 
 def assert_close(got, ref, what=""):
-    """Three checks per tensor, all tied to the benchmark spec's bound of 1e-2 (bf16 inputs, fp32 accumulation):
-      max|d| <= 1e-2 max|ref|;   rms(d) <= 5e-3 rms(ref);   |d| <= 1e-2 |ref| + 4e-2 rms(ref) element-wise.
-    The element-wise slack covers what bf16 storage itself costs: an attention weight kept as bf16 carries
-    a relative error of 2^-9, so one dominant key moves an output by up to 2^-9 |v| (|v| up to ~4 rms)."""
+    """Three checks per tensor:
+      max|d| <= 1e-2 max|ref|;   rms(d) <= 5e-3 rms(ref);   |d| <= 1e-2 |ref| + 2e-2 rms(ref) element-wise.
+    Where the element-wise allowance comes from.  Every product is exact in fp32 and an fp32 sum of n <= 13824
+    terms is good to n 2^-24 < 1e-3, so what is left are the bf16 roundings: the output itself (2^-9 |ref|,
+    inside the relative term) and, in attention, the softmax weights, which enter the PV product as bf16 while the
+    row sum is taken from the unrounded values: two independent relative errors of at most 2^-9 per key, uniform,
+    so standard deviation 2^-9 sqrt(2/3) each way.  An output element sum_u p_u v_u then carries an error of standard
+    deviation 2^-9 sqrt(2/3) sqrt(sum_u p_u^2 v_u^2) ~ 1.6e-3 rms(ref) that does not shrink where the element itself
+    is small through cancellation, so it has to be allowed in absolute terms.  Up to 4e6 elements are compared per
+    tensor; the largest of that many normal deviates is about sqrt(2 ln 4e6) = 5.5 standard deviations = 0.9e-2
+    rms(ref).  The allowance is twice that expected maximum.  (The SGMV path rounds the LoRA term to bf16 before
+    the add: 2^-9 of a term that is a tenth of y, far inside.)"""
     got = np.asarray(got, dtype=np.float64)
     ref = np.asarray(ref, dtype=np.float64)
     assert got.shape == ref.shape, (what, got.shape, ref.shape)
@@ -21,9 +34,16 @@ def assert_close(got, ref, what=""):
     d = np.abs(got - ref)
     scale = np.abs(ref).max()
     rms = np.sqrt(np.mean(ref * ref))
+    if os.environ.get("FL_TOL_REPORT"):
+        need = float(((d - REL * np.abs(ref)) / max(rms, 1e-30)).max())
+        key = what.split(" request")[0]
+        if need > _observed.get(key, -1.0):
+            _observed[key] = need
+            with open(os.environ["FL_TOL_REPORT"], "a") as f:
+                f.write(f"{key}\t{need:.5f}\t{d.max() / max(scale, 1e-30):.5f}\t{np.sqrt(np.mean(d * d)) / max(rms, 1e-30):.5f}\n")
     assert d.max() <= REL * max(scale, 1e-30), (what, "max", d.max(), scale)
     assert np.sqrt(np.mean(d * d)) <= 0.5 * REL * max(rms, 1e-30), (what, "rms", np.sqrt(np.mean(d * d)), rms)
-    bad = d > REL * np.abs(ref) + 4 * REL * rms
+    bad = d > REL * np.abs(ref) + SLACK * rms
     assert not bad.any(), (what, "elementwise", int(bad.sum()), d.max(), rms)
 
 

@@ -259,7 +259,7 @@ def _attention_case(H, wl, sm_scale=None, prefill_kernel=0):
         s.close()
 
 
-@pytest.mark.parametrize("kernel", [0, 1, 2])
+@pytest.mark.parametrize("kernel", [0, 1])
 @pytest.mark.parametrize("name", list(REDUCED))
 def test_attention_parity(H, name, kernel):
     _attention_case(H, synth.make_workload(name, **REDUCED[name]), prefill_kernel=kernel)
@@ -268,11 +268,11 @@ def test_attention_parity(H, name, kernel):
 def test_attention_sharp_softmax_rescales_accumulator(H):
     # large logits that keep growing along the keys force the running maximum up tile after tile
     wl = synth.make_workload("prefill7b", n_req=2, len_range=(300, 700))
-    for kernel in (0, 1, 2):
+    for kernel in (0, 1):
         _attention_case(H, wl, sm_scale=1.5, prefill_kernel=kernel)
 
 
-@pytest.mark.parametrize("kernel", [0, 1, 2])
+@pytest.mark.parametrize("kernel", [0, 1])
 def test_attention_edges(H, kernel):
     sh = synth.LayerShape(512, 4, 4)
     # no prefix, one token, ragged tails, a request with no new token, long decode context (several chunks)
@@ -468,6 +468,20 @@ def test_sgmv_qkv_append_equals_projection_then_append(H, name):
             assert torch.equal(tz["q"], want_q)
             got_blocks = fl.device_block_bytes(s.pool, s.block_bytes, blocks)
             assert np.array_equal(got_blocks, want_blocks), (name, drop_some)
+            # and against the oracle itself: q, and the K, V rows read back out of the pool blocks
+            lid = mixed if drop_some else ids
+            x = wl.x("q")
+            want = {m: lora_project(wl.y_base(m), x, seg, lid, oracle_adapters(wl, m), wl.scale) for m in "qkv"}
+            assert_close(H.dev_to_f32(tz["q"]), want["q"], f"{name}/fused q")
+            pos_of = {b: k for k, b in enumerate(blocks)}
+            gb = got_blocks.view(np.uint16).reshape(len(blocks), 2, sh.n_kv_heads, sh.block_tokens, 128)
+            for i in range(wl.n_req):
+                lo, hi = int(wl.req_indptr[i]), int(wl.req_indptr[i + 1])
+                pos = int(wl.prefix_lens[i]) + np.arange(hi - lo)
+                blk = np.array([pos_of[tables[i][e]] for e in pos // sh.block_tokens])
+                rows = op.bf16_bits_to_f64(gb[blk, :, :, pos % sh.block_tokens, :])       # [n, 2, n_kv, 128]
+                assert_close(rows[:, 0].reshape(hi - lo, -1), want["k"][lo:hi], f"{name}/fused K in pool")
+                assert_close(rows[:, 1].reshape(hi - lo, -1), want["v"][lo:hi], f"{name}/fused V in pool")
             # k, v inputs are left as they were
             assert np.array_equal(H.dev_to_f32(tz["k"]), wl.y_base("k")) and np.array_equal(H.dev_to_f32(tz["v"]), wl.y_base("v"))
     finally:

@@ -79,6 +79,43 @@ def test_lora_block_counts_match_hand_arithmetic():
                 spans.add(key)
 
 
+def test_adapter_bytes_by_hand_on_the_gqa_rank64_shape():
+    """Placement of single adapter elements worked out by hand (Section 4.3: adapters are cut along the rank
+    dimension into rows that share blocks with KV).  34B-class layer: hidden 8192, 64 query / 8 KV heads,
+    rank 64, blocks of 64 KiB = 32768 bf16 values.  Row order A_q B_q A_k B_k A_v B_v A_o B_o; row p of A is
+    A[:, p], row p of B is B[p, :].
+      width 8192 (4 rows per block):  A_q rows 0..63, B_q 64..127, A_k 128..191, A_v 192..255, A_o 256..319,
+                                      B_o 320..383  -> 96 blocks, table entries 0..95
+      width 1024 (32 rows per block): B_k rows 0..63, B_v 64..127 -> 4 blocks, table entries 96..99
+      A_k[5, 3]    = row 128 + 3 = 131  -> entry 131 // 4 = 32,     value index (131 % 4) * 8192 + 5    = 24581
+      B_o[7, 100]  = row 320 + 7 = 327  -> entry 327 // 4 = 81,     value index (327 % 4) * 8192 + 100  = 24676
+      B_v[9, 1000] = row 64 + 9 = 73    -> entry 96 + 73 // 32 = 98, value index (73 % 32) * 1024 + 1000 = 10216
+      A_q[8191, 63] = row 63            -> entry 15,                value index 3 * 8192 + 8191 = 32767 (last of its block)
+      B_k[0, 0]    = row 0 of its class -> entry 96,                value index 0"""
+    shp = synth.LayerShape(8192, 64, 8)
+    assert shp.block_bytes == 65536
+    mats = [(i, o) for _, i, o in shp.mats]
+    rank = 64
+    rs = synth.Stream(12, "pin")
+    A = [synth.bf16_bits(rs.normal((i, rank), 0.5)) for i, _ in mats]
+    B = [synth.bf16_bits(rs.normal((rank, o), 0.5)) for _, o in mats]
+    pool = op.PoolModel(shp.block_bytes, 8, 128)
+    table = pool.alloc(100, host=True)[::-1]          # entry e -> host block 99 - e
+    pool.pack_lora(table, rank, mats, A, B, host=True)
+    q, k, v, o = 0, 1, 2, 3
+    by_hand = [(32, 24581, A[k][5, 3]), (81, 24676, B[o][7, 100]), (98, 10216, B[v][9, 1000]),
+               (15, 32767, A[q][8191, 63]), (96, 0, B[k][0, 0])]
+    for entry, idx, want in by_hand:
+        assert pool.block(99 - entry, host=True).view(np.uint16)[idx] == want, (entry, idx)
+    # a whole row, so that a rotation inside the row would show as well: row 2 of B_q = entry (64 + 2) // 4, slot 2
+    got = pool.block(99 - 16, host=True).view(np.uint16)[2 * 8192:3 * 8192]
+    assert np.array_equal(got, B[q][2, :])
+    # and the read side on its own: the gather returns A_k, not its transpose or another matrix
+    a_k, b_k = pool.read_lora(table, rank, mats, k, host=True)
+    assert a_k.shape == (8192, 64) and b_k.shape == (64, 1024)
+    assert a_k[5, 3] == synth.bf16_to_f32(A[k][5:6, 3])[0] and b_k[9, 1000] == synth.bf16_to_f32(B[k][9:10, 1000])[0]
+
+
 def _small_pool(n_blocks=40, n_kv=2, d=8, bt=4):
     return op.PoolModel(bt * 2 * n_kv * d * 2, n_blocks, 16), n_kv, d, bt
 

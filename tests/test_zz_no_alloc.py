@@ -3,8 +3,10 @@
 An engine that has handed all of its HBM to the block pool (or a plug-in that may not touch the engine's
 memory budget) has no scratch buffer to give fl_lora_sgmv.  fl_lora_sgmv_static uses a fixed array inside
 the library instead.  This test calls it through the C ABI twice in a row, with different inputs, and
-compares each result with what fl_lora_sgmv gives on a caller-provided workspace.  The second call runs
-on whatever the first left in the shared scratch, so a result that depended on stale contents would show.
+compares each result with the CPU oracle and, bit for bit, with what fl_lora_sgmv gives on a caller-provided
+workspace (both run the same kernels).  The second call runs on whatever the first left in the shared scratch,
+so a result that depended on stale contents would show.  Free device memory is read before and after: the calls
+must not change it.
 The file sorts last so that a run that stops at the first failure has already run every other test.
 """
 import numpy as np
@@ -15,7 +17,9 @@ pytestmark = pytest.mark.gpu
 
 from paper_2505_03756_b200 import synth
 
-from _util import assert_close
+from oracle.lora import lora_project
+
+from _util import assert_close, oracle_adapters
 
 
 def test_static_scratch_matches_workspace_variant_twice():
@@ -30,18 +34,30 @@ def test_static_scratch_matches_workspace_variant_twice():
             s.build_batch()
             T = wl.n_tokens
             ws = s.workspace("sgmv", fl.fl_lora_sgmv_workspace(T, 1))
+            seg, ids = wl.segments()
+            bufs = {}
+            for mat in ("q", "o"):                     # every buffer exists before free memory is first read
+                y = H.f32_to_dev(wl.y_base(mat), s.dev)
+                bufs[mat] = (H.f32_to_dev(wl.x(mat), s.dev), y, y.clone())
+            fl.fl_lora_sgmv_static(s.pool, bufs["q"][2].clone(), bufs["q"][0], s.mat_index["q"], s.t_seg_indptr,
+                                   s.t_seg_lora, s.n_seg, T, 0.0)      # the first call on a device looks up the array
+            torch.cuda.synchronize()
+            free_before = torch.cuda.mem_get_info()[0]
             for call, (mat, scale) in enumerate([("q", wl.scale), ("o", -0.75)]):      # two calls in a row
-                tx = H.f32_to_dev(wl.x(mat), s.dev)
-                y_ref = H.f32_to_dev(wl.y_base(mat), s.dev)
-                y_new = y_ref.clone()
+                tx, y_ref, y_new = bufs[mat]
                 fl.fl_lora_sgmv(s.pool, y_ref, tx, s.mat_index[mat], s.t_seg_indptr, s.t_seg_lora, s.n_seg, T,
                                 scale, ws)
                 fl.fl_lora_sgmv_static(s.pool, y_new, tx, s.mat_index[mat], s.t_seg_indptr, s.t_seg_lora, s.n_seg,
                                        T, scale)
-                torch.cuda.synchronize()
+            torch.cuda.synchronize()
+            assert torch.cuda.mem_get_info()[0] == free_before, "the calls changed the amount of free device memory"
+            for call, (mat, scale) in enumerate([("q", wl.scale), ("o", -0.75)]):
+                tx, y_ref, y_new = bufs[mat]
                 ref, got = H.dev_to_f32(y_ref), H.dev_to_f32(y_new)
                 assert not np.array_equal(ref, wl.y_base(mat)), "the projection changed nothing"
-                assert_close(got, ref, f"{wl.name} call {call}")
+                assert np.array_equal(got, ref), f"{wl.name} call {call}: differs from fl_lora_sgmv"
+                want = lora_project(wl.y_base(mat), wl.x(mat), seg, ids, oracle_adapters(wl, mat), scale)
+                assert_close(got, want, f"{wl.name} static call {call}")
             assert s.status()["device_flags"] == 0
         finally:
             s.close()
@@ -59,5 +75,7 @@ def test_static_scratch_rejects_oversized_batches():
         with pytest.raises(fl.FlError) as e:
             fl.fl_lora_sgmv_static(pool, dummy, dummy, 0, dummy, dummy, 1, too_many, 1.0)
         assert e.value.code == fl.FL_ENOMEM
+        # an empty batch is a no-op whatever its other arguments say, as in fl_lora_sgmv
+        fl.fl_lora_sgmv_static(pool, dummy, dummy, 0, dummy, dummy, 0, too_many, 1.0)
     finally:
         fl.fl_pool_destroy(pool)

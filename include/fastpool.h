@@ -220,6 +220,28 @@ int fl_lora_sgmv_static(fl_pool* pool, fl_bf16* y, const fl_bf16* x, int mat_ind
                         const int32_t* seg_indptr, const int32_t* lora_ids, int n_seg, int n_tokens,
                         float scale, fl_stream stream);
 
+/* ---------------------------------------------------------------- base projection with the LoRA branch folded in
+ * Eq. 1 (W' = W + A B) and Eq. 2 (W q + A B q) evaluated in one pass over the output: for every token t,
+ *     y[t, :] = x[t, :] W + scale * (x[t, :] A_i) B_i        (i = adapter of t's segment; none: y = x W)
+ * computed by one tensor-core GEMM whose accumulator also takes the low-rank term before it is stored, so y is
+ * written once and never read (fl_lora_sgmv reads and rewrites a y that another kernel produced).
+ * w: device [d_in, d_out] bf16 row-major, the base weight of projection `mat_index` (shapes as registered with the
+ * adapters: at least one adapter must be registered, FL_EBADID otherwise); x, seg_indptr, lora_ids as in
+ * fl_lora_sgmv; y: device [n_tokens, d_out] bf16, overwritten.  fp32 accumulation over d_in and the rank, the
+ * shrink result x A_i is rounded to bf16 before it meets B_i, one bf16 rounding of the result.
+ * n_seg = 0 is allowed (plain y = x W).  The _multi form runs up to 3 projections that share x (q, k, v) as one
+ * launch: ys, ws and mat_indices are HOST arrays.  workspace: device scratch of at least
+ * fl_lora_linear_workspace(n_tokens, n_mats) bytes, same sharing rule as fl_lora_sgmv.  After one ordinary call
+ * the call only launches kernels on `stream`. */
+size_t fl_lora_linear_workspace(int n_tokens, int n_mats);
+int fl_lora_linear(fl_pool* pool, fl_bf16* y, const fl_bf16* x, const fl_bf16* w, int mat_index,
+                   const int32_t* seg_indptr, const int32_t* lora_ids, int n_seg, int n_tokens,
+                   float scale, void* workspace, size_t workspace_bytes, fl_stream stream);
+int fl_lora_linear_multi(fl_pool* pool, fl_bf16* const* ys, const fl_bf16* x, const fl_bf16* const* ws,
+                         const int* mat_indices, int n_mats, const int32_t* seg_indptr, const int32_t* lora_ids,
+                         int n_seg, int n_tokens, float scale, void* workspace, size_t workspace_bytes,
+                         fl_stream stream);
+
 /* ---------------------------------------------------------------- KV store (Section 4.3: new KV stays in HBM blocks)
  * Writes the new tokens' K and V into the pool.  Request i owns tokens req_indptr[i] .. req_indptr[i+1]
  * of k_new / v_new (device, [n_tokens, n_kv_heads, 128] bf16); its token j goes to logical position

@@ -8,6 +8,8 @@ projections.  In row-vector form with a LoRA scale s, a token row x that uses ad
 Tokens of one batch are grouped into segments, one adapter per segment (the "segmented gather"
 batching the paper cites in Section 2.1).  The base term x W arrives precomputed as y_base.
 
+lora_linear is the same formula with the base term written out: y = x W + s (x A_i) B_i.
+
 Pins: B = 0, scale = 0 or lora id -1 return y_base bit for bit; one adapter over the whole batch
 equals the dense product x (W + s A B) (Eq. 1); linear in s; permuting segments permutes rows; a
 hand-worked integer example.
@@ -31,3 +33,9 @@ def lora_project(y_base, x, seg_indptr, lora_ids, adapters, scale):
         v = x[lo:hi] @ np.asarray(A, dtype=np.float64)          # shrink  [n, r]
         y[lo:hi] += scale * (v @ np.asarray(B, dtype=np.float64))  # expand  [n, d_out]
     return y
+
+
+def lora_linear(x, W, seg_indptr, lora_ids, adapters, scale):
+    """y[t] = x[t] W + scale * (x[t] A_i) B_i (Eq. 1 applied to a row vector); W [d_in, d_out].  Returns float64."""
+    x = np.asarray(x, dtype=np.float64)
+    return lora_project(x @ np.asarray(W, dtype=np.float64), x, seg_indptr, lora_ids, adapters, scale)

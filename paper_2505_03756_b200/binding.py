@@ -88,6 +88,10 @@ _SIGS = {
                                      C.c_float, _vp, C.c_size_t, _vp]),
     "fl_lora_sgmv_qkv_append": (C.c_int, [_vp, _vp, _vp, _vp, _vp, C.c_int, C.c_int, C.c_int, _vp, _vp, C.c_int, C.c_int,
                                           C.c_float, _vp, _vp, _vp, _vp, C.c_int, C.c_int, _vp, C.c_size_t, _vp]),
+    "fl_lora_linear_workspace": (C.c_size_t, [C.c_int, C.c_int]),
+    "fl_lora_linear": (C.c_int, [_vp, _vp, _vp, _vp, C.c_int, _vp, _vp, C.c_int, C.c_int, C.c_float, _vp, C.c_size_t, _vp]),
+    "fl_lora_linear_multi": (C.c_int, [_vp, C.POINTER(_vp), _vp, C.POINTER(_vp), _i32p, C.c_int, _vp, _vp, C.c_int,
+                                       C.c_int, C.c_float, _vp, C.c_size_t, _vp]),
     "fl_kv_append": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, C.c_int, C.c_int, C.c_int, _vp]),
     "fl_paged_attention_workspace": (C.c_size_t, [C.c_int, C.c_int, C.c_int, C.c_int, C.c_int]),
     "fl_paged_attention": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, C.c_int, C.c_int, C.c_int, C.c_int,
@@ -309,6 +313,26 @@ def fl_lora_sgmv_qkv_append(pool, y_q, y_k, y_v, x, mat_q, mat_k, mat_v, seg_ind
                                        _dev(kv_tbl_indptr), _dev(kv_tbl), _dev(prefix_lens), n_req, n_kv_heads,
                                        _dev(workspace), workspace.numel() * workspace.element_size(), _stream(stream)),
            "fl_lora_sgmv_qkv_append")
+
+
+def fl_lora_linear_workspace(n_tokens, n_mats=1):
+    return lib.fl_lora_linear_workspace(n_tokens, n_mats)
+
+
+def fl_lora_linear(pool, y, x, w, mat_index, seg_indptr, lora_ids, n_seg, n_tokens, scale, workspace, stream=None):
+    _check(lib.fl_lora_linear(pool, _dev(y), _dev(x), _dev(w), mat_index, _dev(seg_indptr), _dev(lora_ids), n_seg,
+                              n_tokens, scale, _dev(workspace), workspace.numel() * workspace.element_size(),
+                              _stream(stream)), "fl_lora_linear")
+
+
+def fl_lora_linear_multi(pool, ys, x, ws, mat_indices, seg_indptr, lora_ids, n_seg, n_tokens, scale, workspace,
+                         stream=None):
+    py = (_vp * len(ys))(*[_dev(y) for y in ys])
+    pw = (_vp * len(ws))(*[_dev(w) for w in ws])
+    mi = (C.c_int32 * len(ys))(*[int(m) for m in mat_indices])
+    _check(lib.fl_lora_linear_multi(pool, py, _dev(x), pw, mi, len(ys), _dev(seg_indptr), _dev(lora_ids), n_seg,
+                                    n_tokens, scale, _dev(workspace), workspace.numel() * workspace.element_size(),
+                                    _stream(stream)), "fl_lora_linear_multi")
 
 
 def fl_kv_append(pool, k_new, v_new, req_indptr, kv_tbl_indptr, kv_tbl, prefix_lens, n_req, n_tokens, n_kv_heads,

@@ -12,6 +12,7 @@
 // the instructions spent per byte, not by the contraction.
 #include "mma_utils.cuh"
 #include "pool.cuh"
+#include "sgmv.cuh"
 
 namespace {
 
@@ -597,7 +598,7 @@ int pick_expand_cols(const SgmvArgs& a, int tiles) {
 }
 
 template <int TM, int RMAX>
-int launch_pair(fl_pool* p, SgmvArgs& a, int tiles, int d_out_max, cudaStream_t st) {
+int launch_pair(fl_pool* p, SgmvArgs& a, int tiles, int d_out_max, cudaStream_t st, bool shrink_only) {
   a.expand_cols = pick_expand_cols(a, tiles);
   static bool configured[16] = {};
   const int shrink_smem = SH_STAGES * (TM + RMAX) * 128;
@@ -619,6 +620,7 @@ int launch_pair(fl_pool* p, SgmvArgs& a, int tiles, int d_out_max, cudaStream_t 
   } else {
     FL_CUDA(p, launch_pdl(sgmv_shrink_kernel<TM, RMAX>, dim3(tiles * a.n_mats, a.ksplit), dim3(SG_THREADS), shrink_smem, st, a));
   }
+  if (shrink_only) return FL_OK;       // the caller consumes the partial sums itself
   const dim3 egrid(tiles * a.n_mats, (d_out_max + a.expand_cols - 1) / a.expand_cols);
   // the expand may start while the shrink drains (it waits for the shrink's output inside the kernel)
   FL_CUDA(p, cudaGetLastError());
@@ -653,7 +655,8 @@ struct KvDest {      // where K and V results go when they are appended to the p
 
 int sgmv_common(fl_pool* p, fl_bf16* const* ys, const fl_bf16* x, const int* mat_indices, int n_mats,
                 const int32_t* seg_indptr, const int32_t* lora_ids, int n_seg, int n_tokens,
-                float scale, void* workspace, size_t workspace_bytes, fl_stream stream, const KvDest* kv) {
+                float scale, void* workspace, size_t workspace_bytes, fl_stream stream, const KvDest* kv,
+                sgmv::ShrinkInfo* shrink_only = nullptr) {
   if (!p || n_mats < 1 || n_mats > FL_MAX_MATS || n_seg < 0 || n_tokens < 0 || !ys || !mat_indices) return FL_EINVAL;
   if (n_seg == 0 || n_tokens == 0) return FL_OK;
   if (!x || !seg_indptr || !lora_ids || !workspace) return FL_EINVAL;
@@ -664,7 +667,7 @@ int sgmv_common(fl_pool* p, fl_bf16* const* ys, const fl_bf16* x, const int* mat
   int d_out_max = 0;
   for (int j = 0; j < n_mats; ++j) {
     const int mi = mat_indices[j];
-    if (mi < 0 || mi >= p->n_mats || !ys[j]) return FL_EINVAL;
+    if (mi < 0 || mi >= p->n_mats || (!ys[j] && !shrink_only)) return FL_EINVAL;
     if (p->mats[mi].d_in != p->mats[mat_indices[0]].d_in) return FL_EINVAL;   // the projections share x
     a.y[j] = reinterpret_cast<__nv_bfloat16*>(ys[j]);
     a.mat_index[j] = mi;
@@ -722,22 +725,37 @@ int sgmv_common(fl_pool* p, fl_bf16* const* ys, const fl_bf16* x, const int* mat
     if (shrink_ctas < 592 && need <= workspace_bytes) a.ksplit = 2;
   }
   int rc;
+  const bool so = shrink_only != nullptr;
+  if (so) {
+    shrink_only->ksplit = a.ksplit;
+    shrink_only->rmax = rmax;
+  }
   if (small) {
     const int tiles = n_seg + n_tokens / 16;
-    rc = rmax == 16 ? launch_pair<16, 16>(p, a, tiles, d_out_max, st)
-       : rmax == 32 ? launch_pair<16, 32>(p, a, tiles, d_out_max, st)
-                    : launch_pair<16, 64>(p, a, tiles, d_out_max, st);
+    rc = rmax == 16 ? launch_pair<16, 16>(p, a, tiles, d_out_max, st, so)
+       : rmax == 32 ? launch_pair<16, 32>(p, a, tiles, d_out_max, st, so)
+                    : launch_pair<16, 64>(p, a, tiles, d_out_max, st, so);
   } else {
     const int tiles = n_seg + n_tokens / 64;
-    rc = rmax == 16 ? launch_pair<64, 16>(p, a, tiles, d_out_max, st)
-       : rmax == 32 ? launch_pair<64, 32>(p, a, tiles, d_out_max, st)
-                    : launch_pair<64, 64>(p, a, tiles, d_out_max, st);
+    rc = rmax == 16 ? launch_pair<64, 16>(p, a, tiles, d_out_max, st, so)
+       : rmax == 32 ? launch_pair<64, 32>(p, a, tiles, d_out_max, st, so)
+                    : launch_pair<64, 64>(p, a, tiles, d_out_max, st, so);
   }
   if (prev != p->device && prev >= 0) cudaSetDevice(prev);
   return rc;
 }
 
 }  // namespace
+
+namespace sgmv {
+int shrink(fl_pool* p, const fl_bf16* x, const int* mat_indices, int n_mats, const int32_t* seg_indptr,
+           const int32_t* lora_ids, int n_seg, int n_tokens, void* workspace, size_t workspace_bytes, fl_stream stream,
+           ShrinkInfo* info) {
+  fl_bf16* none[FL_MAX_MATS] = {};
+  return sgmv_common(p, none, x, mat_indices, n_mats, seg_indptr, lora_ids, n_seg, n_tokens, 1.f, workspace,
+                     workspace_bytes, stream, nullptr, info);
+}
+}  // namespace sgmv
 
 extern "C" {
 

@@ -1,4 +1,4 @@
-// tcgen05 / TMEM / TMA / mbarrier wrappers (inline PTX for sm_100a) shared by the tensor-core attention kernels.
+// tcgen05 / TMEM / TMA / mbarrier wrappers (inline PTX for sm_100a) shared by the tensor-core kernels.
 #pragma once
 #include <cuda.h>
 #include <stdint.h>
@@ -44,6 +44,22 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
   asm volatile(
       "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
       ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1) : "memory");
+}
+// AND of a predicate over the `count` threads that meet at named barrier `id` (all of them get the result).
+__device__ __forceinline__ bool group_and(bool mine, int id, int count) {
+  uint32_t r;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t"
+      "setp.ne.u32 p, %1, 0;\n\t"
+      "barrier.cta.red.and.pred q, %2, %3, p;\n\t"
+      "selp.u32 %0, 1, 0, q;\n\t}"
+      : "=r"(r) : "r"(mine ? 1u : 0u), "r"(id), "r"(count) : "memory");
+  return r != 0;
 }
 __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
   asm volatile(

@@ -178,6 +178,14 @@ class Session:
             fl.fl_lora_sgmv_multi(self.pool, ys, x, [self.mat_index[m] for m in mats], self.t_seg_indptr,
                                   self.t_seg_lora, self.n_seg, T, scale, ws, stream)
 
+    def lora_linear(self, ys, x, ws, mats, scale=None, stream=None):
+        """ys[j] = x ws[j] + scale * (x A) B for projections `mats` (names) sharing x; ys are overwritten."""
+        T = self.wl.n_tokens
+        wsp = self.workspace("linear", fl.fl_lora_linear_workspace(T, len(mats)))
+        scale = self.wl.scale if scale is None else scale
+        fl.fl_lora_linear_multi(self.pool, ys, x, ws, [self.mat_index[m] for m in mats], self.t_seg_indptr,
+                                self.t_seg_lora, self.n_seg, T, scale, wsp, stream)
+
     def sgmv_qkv_append(self, y_q, y_k, y_v, x, scale=None, stream=None):
         """q += LoRA term in place; base k, v + LoRA term written straight into the batch's pool blocks."""
         T = self.wl.n_tokens

@@ -198,6 +198,20 @@ class Workload:
         d_out = dict((n, o) for n, _, o in self.shape.mats)[mat]
         return self._normal("ybase_" + mat, (self.n_tokens, d_out), 1.0)
 
+    def weight(self, mat: str) -> np.ndarray:
+        """Base weight W [d_in, d_out] of projection `mat`, N(0, 1/d_in) so that x W has unit variance.  Values are
+        taken from a seeded bank of 2^20 normal draws by a multiplicative hash of the element index (drawing the
+        67 million values of an 8192 x 8192 matrix one by one takes longer than everything else in a test)."""
+        key = ("W", mat)
+        if key not in self._cache:
+            d_in, d_out = dict((n, (i, o)) for n, i, o in self.shape.mats)[mat]
+            bank = round_bf16(Stream(self.seed, "W_" + mat).normal((1 << 20,), 1.0 / np.sqrt(d_in)))
+            k = np.arange(d_in * d_out, dtype=np.uint64)
+            with np.errstate(over="ignore"):
+                k = (k * np.uint64(0x9E3779B97F4A7C15)) >> np.uint64(44)
+            self._cache[key] = bank[k.astype(np.int64)].reshape(d_in, d_out)
+        return self._cache[key]
+
     def adapter(self, lora_id: int, mat: str) -> Tuple[np.ndarray, np.ndarray]:
         """(A [d_in, r], B [r, d_out]) of one adapter's projection, N(0, weight_std^2)."""
         d_in, d_out = dict((n, (i, o)) for n, i, o in self.shape.mats)[mat]

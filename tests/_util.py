@@ -9,6 +9,16 @@ from paper_2505_03756_b200 import synth
 REL = 1e-2      # bound on the error of an output relative to the tensor: bf16 inputs, fp32 accumulation, bf16 output
 SLACK = 2e-2    # element-wise absolute allowance in units of rms(ref), see assert_close
 
+# reduced copies of the five workloads: same layer shapes, sizes the oracle finishes in seconds, still several
+# tiles and ragged tails
+REDUCED = {
+    "tiny": dict(),
+    "prefill7b": dict(n_req=7, len_range=(40, 330)),
+    "decode13b": dict(n_req=24, len_range=(30, 700), n_adapters=12),
+    "gqa34b": dict(n_req=3, len_range=(208, 150), n_adapters=3),
+    "swapstress": dict(n_req=10, len_range=(100, 900), n_adapters=40),
+}
+
 _observed = {}  # what -> largest (|d| - REL |ref|) / rms(ref) seen, written out when FL_TOL_REPORT names a file
 
 
@@ -23,8 +33,10 @@ def assert_close(got, ref, what=""):
     deviation 2^-9 sqrt(2/3) sqrt(sum_u p_u^2 v_u^2) ~ 1.6e-3 rms(ref) that does not shrink where the element itself
     is small through cancellation, so it has to be allowed in absolute terms.  Up to 4e6 elements are compared per
     tensor; the largest of that many normal deviates is about sqrt(2 ln 4e6) = 5.5 standard deviations = 0.9e-2
-    rms(ref).  The allowance is twice that expected maximum.  (The SGMV path rounds the LoRA term to bf16 before
-    the add: 2^-9 of a term that is a tenth of y, far inside.)"""
+    rms(ref).  The allowance is twice that expected maximum.  The LoRA projection has the same structure: the
+    shrink result x A enters the expand product as bf16, one independent 2^-9 rounding per rank term, which shows
+    when y_base = 0 and the LoRA term is the whole output.  Largest values seen on a B200 over the whole suite:
+    1.35e-2 rms(ref) for attention, 1.18e-2 for the projection with y_base = 0."""
     got = np.asarray(got, dtype=np.float64)
     ref = np.asarray(ref, dtype=np.float64)
     assert got.shape == ref.shape, (what, got.shape, ref.shape)

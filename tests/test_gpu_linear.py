@@ -1,0 +1,130 @@
+"""fl_lora_linear: base projection with the LoRA branch folded into the GEMM (Eq. 1, Eq. 2), against the oracle's
+y = x W + s (x A_i) B_i, through the C ABI (run on a B200)."""
+import numpy as np
+import pytest
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+from oracle.lora import lora_linear
+from paper_2505_03756_b200 import synth
+
+from _util import REDUCED, assert_close, oracle_adapters
+
+
+@pytest.fixture(scope="module")
+def H():
+    assert torch.cuda.is_available(), "these tests need a GPU"
+    from paper_2505_03756_b200 import binding, harness
+    return harness
+
+
+def _session(H, wl, **kw):
+    s = H.Session(wl, **kw)
+    s.load_adapters()
+    s.build_batch()
+    return s
+
+
+def _groups(wl):
+    return [["q", "k", "v"], ["o"]] + ([["up"], ["down"]] if wl.shape.inter else [])
+
+
+@pytest.mark.parametrize("name", list(REDUCED))
+def test_lora_linear_parity(H, name):
+    wl = synth.make_workload(name, **REDUCED[name])
+    s = _session(H, wl)
+    try:
+        seg, ids = wl.segments()
+        for grp in _groups(wl):
+            x = wl.x(grp[0])
+            tx = H.f32_to_dev(x, s.dev)
+            tw = [H.f32_to_dev(wl.weight(m), s.dev) for m in grp]
+            d_out = dict((n, o) for n, _, o in wl.shape.mats)
+            ty = [torch.full((wl.n_tokens, d_out[m]), 7.0, dtype=torch.bfloat16, device=s.dev) for m in grp]
+            s.lora_linear(ty, tx, tw, grp)
+            torch.cuda.synchronize()
+            assert s.status()["device_flags"] == 0
+            for m, t in zip(grp, ty):
+                want = lora_linear(x, wl.weight(m), seg, ids, oracle_adapters(wl, m), wl.scale)
+                assert_close(H.dev_to_f32(t), want, f"{name}/linear {m}")
+    finally:
+        s.close()
+
+
+def test_lora_linear_lora_term_alone_and_identities(H):
+    """W = 0 leaves the LoRA term as the whole output (so its own error is measured against itself); scale = 0,
+    no segments and segments without an adapter give the plain product; an unknown adapter only raises the flag."""
+    from paper_2505_03756_b200 import binding as fl
+    wl = synth.make_workload("prefill7b", n_req=6, len_range=(20, 260), n_adapters=4)
+    s = _session(H, wl)
+    try:
+        seg, ids = wl.segments()
+        x = wl.x("q")
+        tx = H.f32_to_dev(x, s.dev)
+        W = wl.weight("q")
+        T = wl.n_tokens
+        ws = s.workspace("linear", fl.fl_lora_linear_workspace(T, 1))
+        y = torch.empty(T, 4096, dtype=torch.bfloat16, device=s.dev)
+        zero_w = torch.zeros(4096, 4096, dtype=torch.bfloat16, device=s.dev)
+        fl.fl_lora_linear(s.pool, y, tx, zero_w, 0, s.t_seg_indptr, s.t_seg_lora, s.n_seg, T, wl.scale, ws)
+        want = lora_linear(x, np.zeros_like(W), seg, ids, oracle_adapters(wl, "q"), wl.scale)
+        assert_close(H.dev_to_f32(y), want, "linear/W=0")
+        tw = H.f32_to_dev(W, s.dev)
+        plain = x.astype(np.float64) @ W.astype(np.float64)
+        fl.fl_lora_linear(s.pool, y, tx, tw, 0, s.t_seg_indptr, s.t_seg_lora, s.n_seg, T, 0.0, ws)
+        got0 = H.dev_to_f32(y)
+        assert_close(got0, plain, "linear/scale=0")
+        fl.fl_lora_linear(s.pool, y, tx, tw, 0, s.t_seg_indptr, s.t_seg_lora, 0, T, wl.scale, ws)
+        assert np.array_equal(H.dev_to_f32(y), got0), "no segments: the plain product, bit for bit the same"
+        none = torch.full_like(s.t_seg_lora, -1)
+        fl.fl_lora_linear(s.pool, y, tx, tw, 0, s.t_seg_indptr, none, s.n_seg, T, wl.scale, ws)
+        assert np.array_equal(H.dev_to_f32(y), got0)
+        mixed = ids.copy()
+        mixed[::2] = -1
+        fl.fl_lora_linear(s.pool, y, tx, tw, 0, s.t_seg_indptr, torch.from_numpy(mixed).to(s.dev), s.n_seg, T,
+                          wl.scale, ws)
+        got = H.dev_to_f32(y)
+        assert_close(got, lora_linear(x, W, seg, mixed, oracle_adapters(wl, "q"), wl.scale), "linear/mixed")
+        for k, lid in enumerate(mixed):
+            if lid < 0:
+                assert np.array_equal(got[seg[k]:seg[k + 1]], got0[seg[k]:seg[k + 1]])
+        assert s.status()["device_flags"] == 0
+        bad = torch.full_like(s.t_seg_lora, 3000)
+        fl.fl_lora_linear(s.pool, y, tx, tw, 0, s.t_seg_indptr, bad, s.n_seg, T, wl.scale, ws)
+        assert s.status(clear=True)["device_flags"] & 4
+        assert np.array_equal(H.dev_to_f32(y), got0)
+        # argument checks
+        with pytest.raises(fl.FlError) as e:
+            fl.fl_lora_linear(s.pool, y, tx, tw, 0, s.t_seg_indptr, s.t_seg_lora, s.n_seg, T, 1.0, ws[:256])
+        assert e.value.code == fl.FL_ENOMEM
+        with pytest.raises(fl.FlError):
+            fl.fl_lora_linear(s.pool, y, tx, tw, 9, s.t_seg_indptr, s.t_seg_lora, s.n_seg, T, 1.0, ws)
+    finally:
+        s.close()
+
+
+@pytest.mark.parametrize("hidden,heads,rank", [(320, (4, 4), 5), (200, (2, 1), 24), (1024, (8, 8), 64)])
+def test_lora_linear_odd_shapes_and_ranks(H, hidden, heads, rank):
+    """Output widths that end inside a column tile, an input width that ends inside a k-stage, ranks that are no
+    multiple of 16, one-token segments next to long ones."""
+    shape = synth.LayerShape(hidden, heads[0], heads[1])
+    wl = synth.make_workload("swapstress", n_req=12, len_range=(40, 600), n_adapters=5, shape=shape)
+    wl.ranks[:] = rank
+    s = _session(H, wl)
+    try:
+        seg, ids = wl.segments()
+        for grp in _groups(wl):
+            x = wl.x(grp[0])
+            tx = H.f32_to_dev(x, s.dev)
+            tw = [H.f32_to_dev(wl.weight(m), s.dev) for m in grp]
+            d_out = dict((n, o) for n, _, o in wl.shape.mats)
+            ty = [torch.full((wl.n_tokens, d_out[m]), -3.0, dtype=torch.bfloat16, device=s.dev) for m in grp]
+            s.lora_linear(ty, tx, tw, grp)
+            torch.cuda.synchronize()
+            for m, t in zip(grp, ty):
+                want = lora_linear(x, wl.weight(m), seg, ids, oracle_adapters(wl, m), wl.scale)
+                assert_close(H.dev_to_f32(t), want, f"linear {hidden}/{rank}/{m}")
+        assert s.status()["device_flags"] == 0
+    finally:
+        s.close()

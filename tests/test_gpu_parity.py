@@ -13,7 +13,7 @@ from oracle.layer import attention_layer_step
 from oracle.lora import lora_project
 from paper_2505_03756_b200 import synth
 
-from _util import assert_close, oracle_adapters, oracle_context, replay_trace
+from _util import REDUCED, assert_close, oracle_adapters, oracle_context, replay_trace
 
 
 @pytest.fixture(scope="module")
@@ -28,15 +28,6 @@ def _session(H, wl, **kw):
     s.load_adapters()
     s.build_batch()
     return s
-
-
-REDUCED = {
-    "tiny": dict(),
-    "prefill7b": dict(n_req=7, len_range=(40, 330)),
-    "decode13b": dict(n_req=24, len_range=(30, 700), n_adapters=12),
-    "gqa34b": dict(n_req=3, len_range=(208, 150), n_adapters=3),
-    "swapstress": dict(n_req=10, len_range=(100, 900), n_adapters=40),
-}
 
 
 # ------------------------------------------------------------------ a1: allocator, tables, adapter bytes

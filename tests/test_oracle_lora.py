@@ -1,7 +1,7 @@
 """Pins for oracle/lora.py (O1): special cases, the dense closed form of Eq. 1, a hand-worked example."""
 import numpy as np
 
-from oracle.lora import lora_project
+from oracle.lora import lora_linear, lora_project
 from paper_2505_03756_b200 import synth
 
 
@@ -83,3 +83,22 @@ def test_empty_inputs():
     assert lora_project(yb[:0], x[:0], [0], [], ad, 2.0).shape == (0, yb.shape[1])
     got = lora_project(yb, x, [0, 0, 11], [1, 2], ad, 2.0)   # an empty segment in front
     np.testing.assert_allclose(got, lora_project(yb, x, [0, 11], [2], ad, 2.0))
+
+
+def test_linear_with_base_weight_by_hand_and_against_the_updated_weight():
+    # x = [1, 2], W = [[1, 2, 3], [4, 5, 6]] -> xW = [9, 12, 15]; A = [[1], [1]] -> xA = [3]; B = [[1, 0, -1]];
+    # s = 2 -> y = [9 + 6, 12, 15 - 6]
+    y = lora_linear(np.array([[1., 2.]]), np.array([[1., 2., 3.], [4., 5., 6.]]), [0, 1], [0],
+                    {0: (np.array([[1.], [1.]]), np.array([[1., 0., -1.]]))}, 2.0)
+    assert y.tolist() == [[15., 12., 9.]]
+    # a segment without an adapter is the plain product
+    y = lora_linear(np.array([[1., 2.]]), np.array([[1., 2., 3.], [4., 5., 6.]]), [0, 1], [-1], {}, 2.0)
+    assert y.tolist() == [[9., 12., 15.]]
+    # Eq. 1 per segment: rows of adapter i see W + s A_i B_i
+    x, _, ad, seg, ids = _case(seed=6)
+    W = synth.Stream(9, "w").normal((x.shape[1], 40)).astype(np.float64)
+    got = lora_linear(x, W, seg, ids, ad, 0.5)
+    for s_, lid in enumerate(ids):
+        A, B = (m.astype(np.float64) for m in ad[int(lid)])
+        rows = slice(seg[s_], seg[s_ + 1])
+        np.testing.assert_allclose(got[rows], x[rows].astype(np.float64) @ (W + 0.5 * (A @ B)), rtol=1e-12, atol=1e-12)

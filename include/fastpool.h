@@ -351,8 +351,11 @@ int fl_swapper_decide(const fl_node_stat* nodes, int n, const fl_swap_params* pr
  * node used longest ago leaves first, the node used last enters first) instead of Eq. 6.  FL_POLICY_NO_LORA_REWARD:
  * the coefficient of Eq. 4 is 1 for every node.  policy = 0 is fl_swapper_decide.  Unlike fl_swapper_decide,
  * blocks_used may exceed blocks_total: a caller that needs room for blocks it has not allocated yet adds them to
- * blocks_used, and the swap-out list then frees enough for usage to fall back to `upper`. */
-enum { FL_POLICY_LRU = 1, FL_POLICY_NO_LORA_REWARD = 2 };
+ * blocks_used, and the swap-out list then frees enough for usage to fall back to `upper`.
+ * FL_POLICY_ONLY_LORA / FL_POLICY_ONLY_KV: only nodes of that kind are offered; with blocks_used and blocks_total
+ * those of one partition this is the tick of a statically partitioned HBM (Section 2.2: a fixed share for LoRAs,
+ * the rest for KV caches, the setting the unified pool replaces). */
+enum { FL_POLICY_LRU = 1, FL_POLICY_NO_LORA_REWARD = 2, FL_POLICY_ONLY_LORA = 4, FL_POLICY_ONLY_KV = 8 };
 int fl_swapper_decide_policy(const fl_node_stat* nodes, int n, const fl_swap_params* prm, uint32_t blocks_used,
                              uint32_t blocks_total, uint32_t policy, int32_t* order, int* n_order, int* direction);
 
@@ -393,7 +396,9 @@ int fl_tree_stats(fl_tree* tree, fl_node_stat* out, int cap, int* n_nodes, doubl
 int fl_tree_set_location(fl_tree* tree, int32_t node, int in_hbm, const uint32_t* blocks, uint32_t n_blocks);
 /* FL_TREE_OPT_DEPENDENCY (default 1).  0 = the ablation of Section 6 "Effectiveness of the Cache Manager": usage
  * dependencies are ignored, fl_tree_stats offers every node as a candidate and fl_tree_set_location refuses no
- * move, so KV nodes can stay in HBM below a node that has left ("invalid KV caches").
+ * move, so KV nodes can stay in HBM below a node that has left ("invalid KV caches").  2 = adapters and KV caches
+ * managed apart (the static partition of Section 2.2): LoRA nodes are always offered and never refused, KV nodes keep
+ * the leaf / root rules among themselves, a KV node right below its adapter's node counting as a root.
  * fl_tree_invalid counts them: *hbm_kv = KV nodes in HBM, *invalid_kv = those with an ancestor (their adapter
  * included) outside HBM. */
 enum { FL_TREE_OPT_DEPENDENCY = 0 };
@@ -402,6 +407,38 @@ int fl_tree_invalid(fl_tree* tree, uint32_t* invalid_kv, uint32_t* hbm_kv);
 /* Verifies that every node in HBM has its parent in HBM ("all KV caches that reside in the HBM are valid").
  * FL_EBADID and *first_bad (may be NULL) on a violation. */
 int fl_tree_check(fl_tree* tree, int32_t* first_bad);
+
+/* ---------------------------------------------------------------- trace replay (Sections 4.2, 5.3, 6; host code)
+ * Replays a trace of queries through the dependency tree and the cache swapper with HBM reduced to `capacity`
+ * blocks, and counts what the policy achieves.  Per query: match (Section 4.2); count the matched blocks that are
+ * usable (adapter and whole prefix in HBM) or an adapter cold start; swap in what the query needs, root first, asking
+ * the swapper for room with the query's own nodes held back (Section 5.3); insert the new KV below the matched
+ * prefix; every tick_every queries one monitor tick and a sample of the share of KV nodes in HBM that an absent
+ * ancestor makes unusable.  Query k arrives at t0 + k * dt seconds.  Adapters are nodes of lora_blocks blocks that
+ * start in host memory.  variant: the full policy, or one of the ablations of Section 6 (FL_REPLAY_WOS: LRU instead
+ * of Eq. 6; FL_REPLAY_WOL: Eq. 4 = 1; FL_REPLAY_WOM: dependencies ignored), or FL_REPLAY_STATIC: HBM cut into a
+ * LoRA partition of floor(lora_share * capacity) blocks and a KV partition of the rest, each run by LRU on demand,
+ * no tick moves (Section 2.2; the paper quotes a LoRA share of 0.2).
+ * Query k uses adapter event_lora[k] and the tokens tokens[event_indptr[k] .. event_indptr[k+1]) (host pointers).
+ * FL_ENOMEM: a query does not fit the pool even after everything offered has left. */
+enum { FL_REPLAY_FULL = 0, FL_REPLAY_WOS = 1, FL_REPLAY_WOL = 2, FL_REPLAY_WOM = 3, FL_REPLAY_STATIC = 4 };
+typedef struct {
+  int32_t variant;
+  uint32_t capacity;          /* HBM blocks */
+  int32_t block_tokens;
+  uint32_t lora_blocks;       /* size of every adapter */
+  int32_t tick_every;
+  int32_t batch_size;         /* BS of Eq. 3 */
+  size_t block_bytes;
+  double link_bytes_per_s, upper, lower, t0, dt;
+  double lora_share;          /* FL_REPLAY_STATIC only */
+} fl_replay_config;
+typedef struct {
+  uint64_t asked_blocks, hit_blocks, lora_cold, swapped_in, swapped_out, used_blocks, n_nodes;
+  uint32_t n_samples;         /* monitor ticks taken; invalid_samples[0 .. min(n_samples, cap)) were written */
+} fl_replay_result;
+int fl_cache_replay(const fl_replay_config* cfg, int n_lora, const int32_t* event_lora, const int32_t* event_indptr,
+                    const int32_t* tokens, int n_events, fl_replay_result* out, double* invalid_samples, uint32_t cap);
 
 #ifdef __cplusplus
 }

@@ -47,12 +47,13 @@ def evaluate(nodes, prm):
     return out
 
 
-def decide(nodes, prm, blocks_used, blocks_total, lru=False, lora_reward=True):
+def decide(nodes, prm, blocks_used, blocks_total, lru=False, lora_reward=True, only_kind=None):
     """One monitor tick.  Returns (direction, ordered node indices): -1 swap-out, +1 swap-in, 0 nothing.
 
     The paper's ablations (Section 6): lru=True replaces the cost model by last use alone (the variant "WOS":
     least recently used leaves first, most recently used enters first); lora_reward=False drops the coefficient of
-    Eq. 4 (the variant "WOL").  blocks_used may include blocks the caller is about to allocate."""
+    Eq. 4 (the variant "WOL").  blocks_used may include blocks the caller is about to allocate.  only_kind = LORA or KV
+    offers nodes of that kind alone (a partition that holds one kind, Section 2.2)."""
     usage = blocks_used / blocks_total
     if prm["lower"] <= usage <= prm["upper"]:
         return 0, []
@@ -61,7 +62,8 @@ def decide(nodes, prm, blocks_used, blocks_total, lru=False, lora_reward=True):
     else:
         ev = evaluate(nodes, prm if lora_reward else dict(prm, low_lora=0.0))
     out = usage > prm["upper"]
-    cand = [i for i, nd in enumerate(nodes) if nd["candidate"] and bool(nd["in_hbm"]) == out]
+    cand = [i for i, nd in enumerate(nodes) if nd["candidate"] and bool(nd["in_hbm"]) == out and
+            (only_kind is None or nd["kind"] == only_kind)]
     cand.sort(key=lambda i: (ev[i] if out else -ev[i], i))
     used, order = float(blocks_used), []
     for i in cand:

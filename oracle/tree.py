@@ -25,7 +25,10 @@ class TreeError(Exception):
 class Tree:
     def __init__(self, bt, dependency=True):
         """dependency=False is the paper's ablation "WOM" (Section 6): usage dependencies are ignored, every node is
-        a swap candidate and no move is refused, so KV nodes may stay in HBM below a node that has left."""
+        a swap candidate and no move is refused, so KV nodes may stay in HBM below a node that has left.
+        dependency="kv" models a cache whose adapters and KV caches are managed apart from each other (the static
+        partition of Section 2.2): adapters come and go freely whatever lies below them, KV nodes keep the leaf /
+        root rules among themselves (a KV node right below its adapter's node counts as a root)."""
         self.bt = bt
         self.dependency = dependency
         self.nodes = []          # dicts: parent, kind, lora_id, in_hbm, visits, last_use_s, blocks, children {label: id}
@@ -88,8 +91,11 @@ class Tree:
         """Per node: dict for the swapper (candidate flags per Section 4.2), plus total visits and adapters in HBM."""
         out = []
         for i, nd in enumerate(self.nodes):
-            if not self.dependency:
+            if not self.dependency or (self.dependency == "kv" and nd["kind"] == LORA):
                 cand = True
+            elif self.dependency == "kv" and not nd["in_hbm"]:
+                par = self.nodes[nd["parent"]]
+                cand = par["kind"] == LORA or par["in_hbm"]
             elif nd["in_hbm"]:
                 cand = self._hbm_children(i) == 0
             else:
@@ -104,9 +110,11 @@ class Tree:
         in_hbm = bool(in_hbm)
         if len(blocks) != len(nd["blocks"]) or in_hbm == nd["in_hbm"]:
             raise TreeError("bad move")
-        if self.dependency and not in_hbm and self._hbm_children(n) != 0:
+        free = not self.dependency or (self.dependency == "kv" and nd["kind"] == LORA)
+        if not free and not in_hbm and self._hbm_children(n) != 0:
             raise TreeError("only a leaf of the HBM part may leave")
-        if self.dependency and in_hbm and nd["parent"] >= 0 and not self.nodes[nd["parent"]]["in_hbm"]:
+        if not free and in_hbm and nd["parent"] >= 0 and not self.nodes[nd["parent"]]["in_hbm"] and \
+                not (self.dependency == "kv" and self.nodes[nd["parent"]]["kind"] == LORA):
             raise TreeError("only a root of the host part may enter")
         nd["in_hbm"] = in_hbm
         nd["blocks"] = [int(b) for b in blocks]

@@ -43,6 +43,19 @@ class fl_swap_params(C.Structure):
                 ("block_bytes", C.c_size_t), ("link_bytes_per_s", C.c_double), ("upper", C.c_double), ("lower", C.c_double)]
 
 
+class fl_replay_config(C.Structure):
+    _fields_ = [("variant", C.c_int32), ("capacity", C.c_uint32), ("block_tokens", C.c_int32), ("lora_blocks", C.c_uint32),
+                ("tick_every", C.c_int32), ("batch_size", C.c_int32), ("block_bytes", C.c_size_t),
+                ("link_bytes_per_s", C.c_double), ("upper", C.c_double), ("lower", C.c_double), ("t0", C.c_double),
+                ("dt", C.c_double), ("lora_share", C.c_double)]
+
+
+class fl_replay_result(C.Structure):
+    _fields_ = [("asked_blocks", C.c_uint64), ("hit_blocks", C.c_uint64), ("lora_cold", C.c_uint64),
+                ("swapped_in", C.c_uint64), ("swapped_out", C.c_uint64), ("used_blocks", C.c_uint64),
+                ("n_nodes", C.c_uint64), ("n_samples", C.c_uint32)]
+
+
 class fl_status(C.Structure):
     _fields_ = [("device_flags", C.c_uint32), ("blocks_used", C.c_uint32), ("blocks_free", C.c_uint32),
                 ("host_blocks_used", C.c_uint32), ("host_blocks_free", C.c_uint32), ("lora_blocks", C.c_uint32),
@@ -116,6 +129,8 @@ _SIGS = {
     "fl_tree_check": (C.c_int, [_vp, _i32p]),
     "fl_tree_set_option": (C.c_int, [_vp, C.c_int, C.c_int]),
     "fl_tree_invalid": (C.c_int, [_vp, _u32p, _u32p]),
+    "fl_cache_replay": (C.c_int, [C.POINTER(fl_replay_config), C.c_int, _vp, _vp, _vp, C.c_int,
+                                  C.POINTER(fl_replay_result), _vp, C.c_uint32]),
     "fl_swapper_decide_policy": (C.c_int, [C.POINTER(fl_node_stat), C.c_int, C.POINTER(fl_swap_params), C.c_uint32,
                                            C.c_uint32, C.c_uint32, _vp, C.POINTER(C.c_int), C.POINTER(C.c_int)]),
     "fl_expected_lora_demand": (C.c_int, [_vp, C.c_int, C.c_int, C.POINTER(C.c_double)]),
@@ -449,8 +464,30 @@ def fl_swapper_decide(nodes, prm, blocks_used, blocks_total):
     return d.value, order[:n.value].tolist()
 
 
-FL_POLICY_LRU, FL_POLICY_NO_LORA_REWARD = 1, 2
+FL_POLICY_LRU, FL_POLICY_NO_LORA_REWARD, FL_POLICY_ONLY_LORA, FL_POLICY_ONLY_KV = 1, 2, 4, 8
 FL_TREE_OPT_DEPENDENCY = 0
+FL_REPLAY_FULL, FL_REPLAY_WOS, FL_REPLAY_WOL, FL_REPLAY_WOM, FL_REPLAY_STATIC = 0, 1, 2, 3, 4
+
+
+def fl_cache_replay(events, n_lora, variant, capacity, bt=16, lora_blocks=2, tick_every=8, batch_size=8,
+                    block_bytes=65536, link_bytes_per_s=50e9, upper=0.95, lower=0.70, t0=1.0, dt=0.05, lora_share=0.2):
+    """events: [(lora_id, tokens), ...].  Returns the counters of fl_replay_result plus the invalid-KV samples."""
+    cfg = fl_replay_config(variant, capacity, bt, lora_blocks, tick_every, batch_size, block_bytes, link_bytes_per_s,
+                           upper, lower, t0, dt, lora_share)
+    lora = np.ascontiguousarray([e[0] for e in events], dtype=np.int32)
+    indptr = np.zeros(len(events) + 1, dtype=np.int32)
+    for k, e in enumerate(events):
+        indptr[k + 1] = indptr[k] + len(e[1])
+    tok = np.ascontiguousarray(np.concatenate([np.asarray(e[1], dtype=np.int32) for e in events])
+                               if len(events) else np.zeros(0, np.int32), dtype=np.int32)
+    res = fl_replay_result()
+    cap = len(events) // max(1, tick_every) + 1
+    samples = np.zeros(cap, dtype=np.float64)
+    _check(lib.fl_cache_replay(C.byref(cfg), n_lora, lora.ctypes.data, indptr.ctypes.data, tok.ctypes.data, len(events),
+                               C.byref(res), samples.ctypes.data, cap), "fl_cache_replay")
+    out = {k: int(getattr(res, k)) for k, _ in fl_replay_result._fields_ if k != "n_samples"}
+    out["invalid_samples"] = samples[:res.n_samples].tolist()
+    return out
 
 
 def fl_swapper_decide_policy(nodes, prm, blocks_used, blocks_total, policy):

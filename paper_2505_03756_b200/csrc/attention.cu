@@ -41,9 +41,16 @@ __device__ __forceinline__ int block_excl_scan(int val, int* sh, int& total) {
 
 __global__ void __launch_bounds__(256) attn_plan_kernel(const AttnArgs a, int chunk, int qt) {
   __shared__ int sh[8];
+  __shared__ int hist[64], cursor[64];
   pdl_wait();                 // the lists may still be read, and the request arrays written, by the kernel before
   pdl_launch_dependents();    // the prefill kernel sets itself up (barriers, TMEM) while this single CTA plans
   const int group = a.n_q / a.n_kv;
+  if (threadIdx.x < 64) hist[threadIdx.x] = 0;
+  __syncthreads();
+  // Prefill requests are ordered by context length (in 128-key steps), longest first, so that the CTAs that take work
+  // from the list finish together; the tiles of one request stay next to each other (its later tiles first), so the
+  // units that read the same K/V pages run at about the same time and the second reader finds them in L2.
+  auto key_of = [&](int i) { return min(63, (a.prefix_lens[i] + a.new_lens[i] + 127) / 128); };
   int base_p = 0, base_d = 0;
   for (int i0 = 0; i0 < a.n_req; i0 += 256) {
     const int i = i0 + threadIdx.x;
@@ -58,32 +65,20 @@ __global__ void __launch_bounds__(256) attn_plan_kernel(const AttnArgs a, int ch
       }
     }
     int tot_p, tot_d;
-    const int off_p = base_p + block_excl_scan(tiles, sh, tot_p);
+    block_excl_scan(tiles, sh, tot_p);
     const int off_d = base_d + block_excl_scan(chunks, sh, tot_d);
     if (i < a.n_req) {
       // a request whose chunks do not all fit in the list (contexts longer than the caller's n_tbl covers) gets no
       // output: the chunks that did fit only write partial slots inside the workspace, and the merge, which would
       // read all of them, skips the request (the overflow raises FLAG_BAD_POS below)
       a.req_info[i] = make_int4(off_d, off_d + chunks > a.max_decode ? 0 : chunks, dec ? 1 : 0, 0);
-      for (int t = 0; t < tiles; ++t)
-        if (off_p + t < a.max_prefill) a.prefill_tmp[off_p + t] = make_int2(i, t * qt);
+      if (tiles > 0) atomicAdd(&hist[key_of(i)], tiles);
       for (int c = 0; c < chunks; ++c)
         if (off_d + c < a.max_decode) a.decode_list[off_d + c] = make_int2(i, c);
     }
     base_p += tot_p;
     base_d += tot_d;
   }
-  // Prefill tiles go out longest first (counting sort on the number of 128-key tiles a tile reads), so that the
-  // CTAs that take work from the list finish together; tiles of equal length land in no particular order.
-  __shared__ int hist[64], cursor[64];
-  const int n_p = min(base_p, a.max_prefill);
-  if (threadIdx.x < 64) hist[threadIdx.x] = 0;
-  __syncthreads();
-  auto key_of = [&](int2 it) {
-    const int kv_end = min(a.prefix_lens[it.x] + a.new_lens[it.x], a.prefix_lens[it.x] + it.y + qt);
-    return min(63, (kv_end + 127) / 128);
-  };
-  for (int idx = threadIdx.x; idx < n_p; idx += 256) atomicAdd(&hist[key_of(a.prefill_tmp[idx])], 1);
   __syncthreads();
   if (threadIdx.x == 0) {
     int start = 0;
@@ -93,9 +88,13 @@ __global__ void __launch_bounds__(256) attn_plan_kernel(const AttnArgs a, int ch
     }
   }
   __syncthreads();
-  for (int idx = threadIdx.x; idx < n_p; idx += 256) {
-    const int2 it = a.prefill_tmp[idx];
-    a.prefill_list[atomicAdd(&cursor[key_of(it)], 1)] = it;
+  for (int i = threadIdx.x; i < a.n_req; i += 256) {
+    const int n = a.new_lens[i];
+    if (n <= 0 || n * group <= DEC_ROWS) continue;
+    const int tiles = (n + qt - 1) / qt;
+    const int first = atomicAdd(&cursor[key_of(i)], tiles);
+    for (int t = 0; t < tiles; ++t)
+      if (first + t < a.max_prefill) a.prefill_list[first + t] = make_int2(i, (tiles - 1 - t) * qt);
   }
   if (threadIdx.x == 0) {
     if (base_p > a.max_prefill || base_d > a.max_decode) atomicOr(a.pv.flags, (uint32_t)FLAG_BAD_POS);
@@ -471,7 +470,7 @@ int pick_chunk(int n_tbl, int n_kv) {
 size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 
 struct WsLayout {
-  size_t hdr, prefill_list, prefill_tmp, decode_list, req_info, part_o, part_ml, total;
+  size_t hdr, prefill_list, decode_list, req_info, part_o, part_ml, total;
   int max_prefill, max_decode, chunk;
 };
 
@@ -483,7 +482,6 @@ WsLayout ws_layout(int n_req, int n_tokens, int n_tbl, int n_kv) {
   size_t off = 0;
   w.hdr = off; off = align256(off + sizeof(PlanHdr));
   w.prefill_list = off; off = align256(off + sizeof(int2) * (size_t)w.max_prefill);
-  w.prefill_tmp = off; off = align256(off + sizeof(int2) * (size_t)w.max_prefill);
   w.decode_list = off; off = align256(off + sizeof(int2) * (size_t)w.max_decode);
   w.req_info = off; off = align256(off + sizeof(int4) * (size_t)n_req);
   w.part_o = off; off = align256(off + sizeof(float) * (size_t)w.max_decode * n_kv * DEC_ROWS * D);
@@ -530,7 +528,6 @@ int fl_paged_attention(fl_pool* p, fl_bf16* out, const fl_bf16* q, const int32_t
   a.scale_log2 = sm_scale * 1.4426950408889634f;
   a.hdr = reinterpret_cast<PlanHdr*>(ws + w.hdr);
   a.prefill_list = reinterpret_cast<int2*>(ws + w.prefill_list);
-  a.prefill_tmp = reinterpret_cast<int2*>(ws + w.prefill_tmp);
   a.decode_list = reinterpret_cast<int2*>(ws + w.decode_list);
   a.req_info = reinterpret_cast<int4*>(ws + w.req_info);
   a.part_o = reinterpret_cast<float*>(ws + w.part_o);

@@ -30,8 +30,7 @@ struct AttnArgs {
   float scale_log2;
   // workspace
   PlanHdr* hdr;
-  int2* prefill_list;   // (request, first query token of the tile inside the request), longest tiles first
-  int2* prefill_tmp;    // the same tiles in request order (scratch of the plan kernel)
+  int2* prefill_list;   // (request, first query token of the tile inside the request), longest requests first
   int2* decode_list;    // (request, chunk)
   int4* req_info;       // (first partial slot, chunks, decode?, 0)
   float* part_o;        // [slot][kv head][16 rows][128]

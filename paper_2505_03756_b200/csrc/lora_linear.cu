@@ -472,12 +472,17 @@ int fl_lora_linear_multi(fl_pool* p, fl_bf16* const* ys, const fl_bf16* x, const
   a.ext_count = ext_count;
   a.ext_list = ext_list;
   a.m_tiles = lw.m_tiles;
-  // few token tiles (a decode batch): narrower column tiles, so that every SM streams a slice of W
+  // Segments of a few tokens each (a decode batch): a 128-token tile would take one LoRA stage per segment, each
+  // for a handful of rows, and y is small next to W.  Then the GEMM computes x W alone (no LoRA stages in the plan)
+  // and the segmented projection adds the LoRA term to y afterwards.
+  const bool hybrid = n_seg > 0 && n_tokens <= 16 * n_seg;
+  if (hybrid) a.n_seg = 0;
+  // few token tiles: narrower column tiles, so that every SM streams a slice of W
   int bn = 256;
   {
     long tiles256 = 0;
     for (int j = 0; j < n_mats; ++j) tiles256 += (long)lw.m_tiles * ((a.d_out[j] + 255) / 256);
-    if (tiles256 < p->sm_count) bn = 64;
+    if (tiles256 < p->sm_count || hybrid) bn = 64;
   }
   a.tile_base[0] = 0;
   for (int j = 0; j < n_mats; ++j) {
@@ -512,6 +517,17 @@ int fl_lora_linear_multi(fl_pool* p, fl_bf16* const* ys, const fl_bf16* x, const
       break;
     }
     sgmv::ShrinkInfo info = {1, p->max_rank <= 16 ? 16 : (p->max_rank <= 32 ? 32 : 64)};
+    if (hybrid) {
+      // y = x W from the GEMM alone, then the segmented projection adds the LoRA term to it
+      a.ksplit = 1;
+      a.rmax = info.rmax;
+      rc = info.rmax == 16 ? launch_linear<64, 16>(p, a, maps, st) : info.rmax == 32 ? launch_linear<64, 32>(p, a, maps, st)
+                                                                                   : launch_linear<64, 64>(p, a, maps, st);
+      if (rc != FL_OK) break;
+      rc = fl_lora_sgmv_multi(p, ys, x, mat_indices, n_mats, seg_indptr, lora_ids, n_seg, n_tokens, scale, wsb + lw.v,
+                              fl_lora_sgmv_workspace(n_tokens, n_mats), stream);
+      break;
+    }
     if (n_seg > 0) {
       rc = sgmv::shrink(p, x, mat_indices, n_mats, seg_indptr, lora_ids, n_seg, n_tokens, wsb + lw.v,
                         fl_lora_sgmv_workspace(n_tokens, n_mats), stream, &info);

@@ -47,7 +47,8 @@ int fl_swapper_decide(const fl_node_stat* nodes, int n, const fl_swap_params* pr
 int fl_swapper_decide_policy(const fl_node_stat* nodes, int n, const fl_swap_params* prm, uint32_t blocks_used,
                              uint32_t blocks_total, uint32_t policy, int32_t* order, int* n_order, int* direction) {
   if (!nodes || !prm || !order || !n_order || !direction || n < 0 || blocks_total == 0) return FL_EINVAL;
-  if (policy & ~(uint32_t)(FL_POLICY_LRU | FL_POLICY_NO_LORA_REWARD)) return FL_EINVAL;
+  if (policy & ~(uint32_t)(FL_POLICY_LRU | FL_POLICY_NO_LORA_REWARD | FL_POLICY_ONLY_LORA | FL_POLICY_ONLY_KV)) return FL_EINVAL;
+  if ((policy & FL_POLICY_ONLY_LORA) && (policy & FL_POLICY_ONLY_KV)) return FL_EINVAL;
   if (!(prm->lower >= 0.0 && prm->lower <= prm->upper && prm->upper <= 1.0)) return FL_EINVAL;
   *n_order = 0;
   *direction = 0;
@@ -66,7 +67,10 @@ int fl_swapper_decide_policy(const fl_node_stat* nodes, int n, const fl_swap_par
   }
   std::vector<int32_t> cand;
   for (int i = 0; i < n; ++i)
-    if (nodes[i].candidate && (nodes[i].in_hbm != 0) == out) cand.push_back(i);
+    if (nodes[i].candidate && (nodes[i].in_hbm != 0) == out &&
+        !((policy & FL_POLICY_ONLY_LORA) && nodes[i].kind != FL_NODE_LORA) &&
+        !((policy & FL_POLICY_ONLY_KV) && nodes[i].kind != FL_NODE_KV))
+      cand.push_back(i);
   // swap-out: ascending benefit; swap-in: descending benefit; equal values keep the lower index first
   std::stable_sort(cand.begin(), cand.end(), [&](int32_t a, int32_t b) { return out ? eval[a] < eval[b] : eval[a] > eval[b]; });
   const double upper_blocks = prm->upper * (double)blocks_total, lower_blocks = prm->lower * (double)blocks_total;

@@ -40,7 +40,8 @@ uint64_t label_hash(const int32_t* tok, int n) {
 
 struct fl_tree {
   int bt = 16;
-  bool dependency = true;   // false: the ablation that ignores usage dependencies (any node may move)
+  int dependency = 1;       // 1: Section 4.2 rules; 0: the ablation that ignores usage dependencies (any node may
+                            // move); 2: adapters move freely, KV nodes keep the rules among themselves
   std::vector<Node> nodes;
   std::unordered_map<int32_t, int32_t> lora_node;   // lora id -> node
   double total_visits = 0.0;
@@ -174,7 +175,13 @@ int fl_tree_stats(fl_tree* t, fl_node_stat* out, int cap, int* n_nodes, double* 
     out[i].kind = nd.kind;
     out[i].in_hbm = nd.in_hbm;
     // swap-out candidates: HBM nodes with no child in HBM; swap-in candidates: host nodes right below HBM (or the root)
-    out[i].candidate = !t->dependency ? 1 : nd.in_hbm ? (nd.hbm_children == 0) : (nd.parent < 0 || t->nodes[nd.parent].in_hbm);
+    if (t->dependency == 0 || (t->dependency == 2 && nd.kind == FL_NODE_LORA))
+      out[i].candidate = 1;
+    else if (nd.in_hbm)
+      out[i].candidate = nd.hbm_children == 0;
+    else
+      out[i].candidate = nd.parent < 0 || t->nodes[nd.parent].in_hbm ||
+                         (t->dependency == 2 && t->nodes[nd.parent].kind == FL_NODE_LORA);
     out[i].n_blocks = (uint32_t)nd.blocks.size();
     out[i].visits = nd.visits;
     out[i].last_use_s = nd.last_use_s;
@@ -188,9 +195,11 @@ int fl_tree_set_location(fl_tree* t, int32_t node, int in_hbm, const uint32_t* b
   in_hbm = in_hbm ? 1 : 0;
   if (n_blocks != nd.blocks.size()) return FL_EINVAL;
   if (in_hbm == nd.in_hbm) return FL_EINVAL;
-  if (t->dependency) {
+  if (t->dependency == 1 || (t->dependency == 2 && nd.kind == FL_NODE_KV)) {
     if (!in_hbm && nd.hbm_children != 0) return FL_EBUSY;                             // only leaves of the HBM part leave
-    if (in_hbm && nd.parent >= 0 && !t->nodes[nd.parent].in_hbm) return FL_EBUSY;     // only roots of the host part enter
+    if (in_hbm && nd.parent >= 0 && !t->nodes[nd.parent].in_hbm &&
+        !(t->dependency == 2 && t->nodes[nd.parent].kind == FL_NODE_LORA))
+      return FL_EBUSY;                                                                // only roots of the host part enter
   }
   nd.in_hbm = in_hbm;
   nd.blocks.assign(blocks, blocks + n_blocks);
@@ -200,8 +209,8 @@ int fl_tree_set_location(fl_tree* t, int32_t node, int in_hbm, const uint32_t* b
 
 int fl_tree_set_option(fl_tree* t, int option, int value) {
   if (!t) return FL_EINVAL;
-  if (option != FL_TREE_OPT_DEPENDENCY) return FL_EINVAL;
-  t->dependency = value != 0;
+  if (option != FL_TREE_OPT_DEPENDENCY || value < 0 || value > 2) return FL_EINVAL;
+  t->dependency = value;
   return FL_OK;
 }
 

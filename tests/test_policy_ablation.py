@@ -65,6 +65,73 @@ def test_invalid_kv_counts_nodes_below_a_departed_ancestor():
     assert strict.invalid() == (0, 2) and all(s["candidate"] == 1 for s in t.stats()[0])
 
 
+# ------------------------------------------------------------------ whole replays worked by hand
+TRACES = {
+    "A": dict(events=[(0, [1, 2, 3, 4]), (1, [5, 6, 7, 8]), (0, [1, 2, 3, 4, 9, 10]), (1, [5, 6, 11, 12]), (0, [1, 2, 3, 4])],
+              kw=dict(n_lora=2, capacity=6, bt=2, lora_blocks=1, tick_every=2)),
+    "B": dict(events=[(0, [1, 2, 3, 4]), (0, [1, 2, 3, 4]), (0, [1, 2, 5, 6]), (1, [7, 8, 9, 10]),
+                      (1, [7, 8, 11, 12, 13, 14]), (0, [1, 2, 3, 4])],
+              kw=dict(n_lora=2, capacity=8, bt=2, lora_blocks=1, tick_every=100)),
+    "C": dict(events=[(0, list(range(1, 9))), (0, list(range(11, 19))), (0, list(range(1, 9)))],
+              kw=dict(n_lora=2, capacity=10, bt=2, lora_blocks=1, tick_every=1, lora_share=0.4)),
+}
+
+
+def _by_hand():
+    import os
+    rows = []
+    for line in open(os.path.join(os.path.dirname(__file__), "golden", "replay_by_hand.txt")):
+        if line.startswith("#") or not line.strip():
+            continue
+        f = line.split()
+        rows.append((f[0], f[1], dict(asked_blocks=int(f[2]), hit_blocks=int(f[3]), lora_cold=int(f[4]),
+                                      swapped_in=int(f[5]), swapped_out=int(f[6]), used_blocks=int(f[7]), n_nodes=int(f[8]),
+                                      invalid_samples=[] if f[9] == "-" else [float(v) for v in f[9].split(",")])))
+    return rows
+
+
+@pytest.mark.parametrize("trace,variant,want", _by_hand())
+def test_oracle_replay_matches_the_hand_worked_traces(trace, variant, want):
+    c = TRACES[trace]
+    kw = dict(c["kw"])
+    n_lora = kw.pop("n_lora")
+    capacity = kw.pop("capacity")
+    got = osim.replay(c["events"], n_lora, variant, capacity, **kw)
+    assert got == want, (trace, variant)
+
+
+@pytest.mark.parametrize("trace,variant,want", _by_hand())
+def test_library_replay_matches_the_hand_worked_traces(trace, variant, want):
+    from paper_2505_03756_b200 import cache_sim
+    c = TRACES[trace]
+    kw = dict(c["kw"])
+    n_lora = kw.pop("n_lora")
+    capacity = kw.pop("capacity")
+    assert cache_sim.replay(c["events"], n_lora, variant, capacity, **kw) == want, (trace, variant)
+
+
+def test_static_partition_switches_by_hand():
+    # adapters and KV apart: an adapter may leave above resident KV (which turns unusable), KV keeps its own leaf rule
+    t = otree.Tree(2, dependency="kv")
+    ln = t.add_lora(0, [0], True, 0.0)
+    k = t.insert(ln, [1, 2, 3, 4], [10, 11], 1.0)
+    st = t.stats()[0]
+    assert [s["candidate"] for s in st] == [1, 0, 1]          # the adapter is offered although n1 lies below it
+    with pytest.raises(otree.TreeError):
+        t.set_location(k[0], False, [0])                      # not a KV leaf
+    t.set_location(ln, False, [1])
+    assert t.invalid() == (2, 2)
+    t.set_location(k[1], False, [2])
+    t.set_location(k[0], False, [3])
+    assert [s["candidate"] for s in t.stats()[0]] == [1, 1, 0]   # n1 may come back below its (absent) adapter, n2 not yet
+    t.set_location(k[0], True, [12])
+    # a partition of one kind: only nodes of that kind are offered, least recently used first
+    nodes = [_node(osw.LORA, 5.0, 1.0), _node(osw.KV, 1.0, 3.0), _node(osw.KV, 1.0, 2.0), _node(osw.LORA, 1.0, 0.5)]
+    prm = dict(PRM, upper=1.0, lower=0.0)
+    assert osw.decide(nodes, prm, 3, 2, lru=True, only_kind=osw.KV) == (-1, [2])
+    assert osw.decide(nodes, prm, 3, 1, lru=True, only_kind=osw.LORA) == (-1, [3, 0])
+
+
 # ------------------------------------------------------------------ the library's switches against the oracle's
 def _random_nodes(seed, n):
     rs = synth.Stream(seed, "ablation-nodes")
@@ -89,8 +156,13 @@ def test_library_policy_flags_match_oracle():
             for flag, kw in ((fl.FL_POLICY_LRU, dict(lru=True)), (fl.FL_POLICY_NO_LORA_REWARD, dict(lora_reward=False)),
                              (0, {})):
                 assert fl.fl_swapper_decide_policy(nodes, prm, used, total, flag) == osw.decide(nodes, prm, used, total, **kw)
+            for flag, kind in ((fl.FL_POLICY_ONLY_LORA, osw.LORA), (fl.FL_POLICY_ONLY_KV, osw.KV)):
+                assert fl.fl_swapper_decide_policy(nodes, prm, used, total, flag | fl.FL_POLICY_LRU) == \
+                    osw.decide(nodes, prm, used, total, lru=True, only_kind=kind)
     with pytest.raises(fl.FlError):
-        fl.fl_swapper_decide_policy(nodes, prm, used, used, 8)                 # unknown flag
+        fl.fl_swapper_decide_policy(nodes, prm, used, used, 16)                # unknown flag
+    with pytest.raises(fl.FlError):
+        fl.fl_swapper_decide_policy(nodes, prm, used, used, 12)                # both kinds at once
     with pytest.raises(fl.FlError):
         fl.fl_swapper_decide(nodes, prm, used + 1, used)                       # the plain tick keeps its range check
     # the tree option
@@ -105,6 +177,23 @@ def test_library_policy_flags_match_oracle():
         fl.fl_tree_set_location(lt, ln, 0, [1])
         assert fl.fl_tree_invalid(lt) == (2, 2)
         assert all(s["candidate"] == 1 for s in fl.fl_tree_stats(lt)[0])
+    finally:
+        fl.fl_tree_destroy(lt)
+    # adapters and KV managed apart: the same moves as in the oracle's pin
+    lt = fl.fl_tree_create(2)
+    try:
+        fl.fl_tree_set_option(lt, fl.FL_TREE_OPT_DEPENDENCY, 2)
+        ln = fl.fl_tree_add_lora(lt, 0, [0], 1, 0.0)
+        k = fl.fl_tree_insert(lt, ln, [1, 2, 3, 4], [10, 11], 1.0)
+        assert [s["candidate"] for s in fl.fl_tree_stats(lt)[0]] == [1, 0, 1]
+        with pytest.raises(fl.FlError):
+            fl.fl_tree_set_location(lt, k[0], 0, [0])
+        fl.fl_tree_set_location(lt, ln, 0, [1])
+        assert fl.fl_tree_invalid(lt) == (2, 2)
+        fl.fl_tree_set_location(lt, k[1], 0, [2])
+        fl.fl_tree_set_location(lt, k[0], 0, [3])
+        assert [s["candidate"] for s in fl.fl_tree_stats(lt)[0]] == [1, 1, 0]
+        fl.fl_tree_set_location(lt, k[0], 1, [12])
     finally:
         fl.fl_tree_destroy(lt)
 
@@ -129,6 +218,8 @@ def test_library_replay_equals_oracle_replay(case, popularity):
         want = osim.replay(events, c["trace"]["n_lora"], variant, **c["sim"])
         assert got == want, (case, popularity, variant)
         res[variant] = want
+    # the fixed split serves fewer cached blocks than the unified pool on every trace of this suite
+    assert res["static"]["hit_blocks"] <= res["full"]["hit_blocks"]
     # with the dependencies kept no KV cache in HBM is ever invalid; without them some are
     for variant in ("full", "wos", "wol"):
         assert max(res[variant]["invalid_samples"]) == 0.0

@@ -110,6 +110,10 @@ int fl_last_cuda_error(fl_pool* pool);
  * = freed blocks keep their contents and fl_block_free touches no device memory. */
 #define FL_OPT_PREFILL_KERNEL 1
 #define FL_OPT_POISON_FREED 2
+/* FL_OPT_SGMV_SHRINK: 0 (default) = batches of long segments run the shrink x A_i on tcgen05 tensor cores (tiles of
+ * 128 tokens, x staged by TMA, adapter rows by cp.async, accumulator in TMEM); 1 = the mma.sync shrink for every
+ * batch.  Same results within rounding (both accumulate in fp32; the order of the sums differs). */
+#define FL_OPT_SGMV_SHRINK 3
 int fl_pool_set_option(fl_pool* pool, int key, int value);
 
 /* ---------------------------------------------------------------- adapters (Section 4.3)

@@ -252,6 +252,7 @@ def fl_last_cuda_error(pool):
 
 FL_OPT_PREFILL_KERNEL = 1
 FL_OPT_POISON_FREED = 2
+FL_OPT_SGMV_SHRINK = 3
 
 
 def fl_pool_set_option(pool, key, value):

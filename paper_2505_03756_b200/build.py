@@ -7,7 +7,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libfastpool.so")
-SOURCES = ["pool.cu", "swap.cu", "sgmv.cu", "attention.cu", "attention_tc2.cu", "tmap.cu", "lora_linear.cu", "swapper.cu", "tree.cu", "cache_sim.cu"]
+SOURCES = ["pool.cu", "swap.cu", "sgmv.cu", "sgmv_tc.cu", "attention.cu", "attention_tc2.cu", "tmap.cu", "lora_linear.cu", "swapper.cu", "tree.cu", "cache_sim.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "--use_fast_math", "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
 

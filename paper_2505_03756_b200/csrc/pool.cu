@@ -250,6 +250,10 @@ int fl_pool_set_option(fl_pool* p, int key, int value) {
     p->prefill_kernel = value;
     return FL_OK;
   }
+  if (key == FL_OPT_SGMV_SHRINK && (value == 0 || value == 1)) {
+    p->sgmv_shrink_kind = value;
+    return FL_OK;
+  }
   if (key == FL_OPT_POISON_FREED && (value == 0 || value == 1)) {
     p->poison_freed = value;
     return FL_OK;

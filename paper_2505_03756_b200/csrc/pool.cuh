@@ -68,6 +68,7 @@ struct fl_pool {
   int last_cuda = 0;
   int sm_count = 148;
   int prefill_kernel = 0;                           // 0: tcgen05 two-tile kernel, 1: mma.sync kernel
+  int sgmv_shrink_kind = 0;                         // 0: tcgen05 shrink for long segments, 1: mma.sync shrink everywhere
   int poison_freed = 0;                             // debugging aid: freed device blocks are filled with NaN patterns
   unsigned char* stage[2] = {nullptr, nullptr};     // contiguous staging areas of the swap path (out, in)
   uint32_t stage_blocks = 0;

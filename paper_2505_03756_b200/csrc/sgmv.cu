@@ -10,11 +10,15 @@
 // small correction of y, so its own 2^-9 roundings stay far below y's final rounding.  Both kernels are
 // bound by memory traffic (x and y rows for long segments, adapter rows for decode-sized segments) and by
 // the instructions spent per byte, not by the contraction.
+#include <algorithm>
 #include "mma_utils.cuh"
 #include "pool.cuh"
 #include "sgmv.cuh"
 
 namespace {
+
+using sgmv::find_tile;
+using sgmv::lora_row;
 
 constexpr int SG_THREADS = 128;
 constexpr int KS = 64;            // d_in elements per shrink pipeline stage (128-byte rows)
@@ -35,6 +39,7 @@ struct SgmvArgs {
   float scale;
   float* v;        // [n_mats][ksplit][n_tokens][RMAX]
   int ksplit;
+  int tc_ksplit;     // slices of d_in for the tcgen05 shrink of long segments (0 = not applicable)
   int expand_cols;   // y columns one expand CTA covers
   int d_out[FL_MAX_MATS];
   // K / V projections whose result goes straight into the requests' pool blocks instead of back into y
@@ -48,43 +53,6 @@ struct SgmvArgs {
   int n_req, n_kv, bt;
 };
 
-// Token tile `tile` (tiles of TM tokens, counted over segments that carry an adapter, or over all segments) -> segment and
-// token range.  Every warp evaluates it redundantly with a warp scan over 32 segments at a time.
-template <int TM>
-__device__ __forceinline__ bool find_tile(const int32_t* __restrict__ seg_indptr, const int32_t* __restrict__ lora_ids,
-                                          int n_seg, int tile, int& seg, int& tok0, int& tok1, bool all_segments = false) {
-  const int lane = threadIdx.x & 31;
-  int base = 0;
-  for (int s0 = 0; s0 < n_seg; s0 += 32) {
-    const int s = s0 + lane;
-    int lo = 0, hi = 0, nt = 0;
-    if (s < n_seg) {
-      lo = seg_indptr[s];
-      hi = seg_indptr[s + 1];
-      if ((all_segments || lora_ids[s] >= 0) && hi > lo) nt = (hi - lo + TM - 1) / TM;
-    }
-    int incl = nt;
-#pragma unroll
-    for (int d = 1; d < 32; d <<= 1) {
-      const int o = __shfl_up_sync(0xffffffffu, incl, d);
-      if (lane >= d) incl += o;
-    }
-    const int total = __shfl_sync(0xffffffffu, incl, 31);
-    if (tile < base + total) {
-      const int first = base + incl - nt;
-      const bool mine = nt > 0 && tile >= first && tile < first + nt;
-      const int src = __ffs(__ballot_sync(0xffffffffu, mine)) - 1;
-      const int k = tile - __shfl_sync(0xffffffffu, first, src);
-      seg = s0 + src;
-      tok0 = __shfl_sync(0xffffffffu, lo, src) + k * TM;
-      tok1 = min(tok0 + TM, __shfl_sync(0xffffffffu, hi, src));
-      return true;
-    }
-    base += total;
-  }
-  return false;
-}
-
 // Eight bf16 sums (round to nearest even each) of two 16-byte chunks.
 __device__ __forceinline__ uint4 add_bf16x8(uint4 a, uint4 b) {
   uint4 r;
@@ -94,20 +62,6 @@ __device__ __forceinline__ uint4 add_bf16x8(uint4 a, uint4 b) {
 #pragma unroll
   for (int i = 0; i < 4; ++i) pr[i] = __hadd2(pa[i], pb[i]);
   return r;
-}
-
-// Start of rank-row `row` of a stream (class table entry tab, first row row0, rows per block rpb, row width).
-__device__ __forceinline__ const unsigned char* lora_row(const PoolView& pv, uint32_t table_off, uint32_t tab,
-                                                         uint32_t row0, uint32_t rpb, int width, int row, bool& ok) {
-  const uint32_t g = row0 + (uint32_t)row;
-  const uint32_t blk = pv.tables[table_off + tab + g / rpb];
-  if (blk >= pv.n_blocks) {
-    atomicOr(pv.flags, (uint32_t)FLAG_BAD_BLOCK);
-    ok = false;
-    return pv.slab;
-  }
-  ok = true;
-  return pv.slab + (size_t)blk * pv.block_bytes + (size_t)(g % rpb) * 2 * (size_t)width;
 }
 
 template <int TM, int RMAX>
@@ -609,7 +563,23 @@ int launch_pair(fl_pool* p, SgmvArgs& a, int tiles, int d_out_max, cudaStream_t 
     FL_CUDA(p, cudaFuncSetAttribute(sgmv_expand_kernel<TM, RMAX, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, expand_smem));
     configured[p->device & 15] = true;
   }
-  if (TM == 64 && RMAX == 16 && a.n_mats == 3) {      // at higher ranks the three accumulators cost too many registers
+  if (TM == 64 && p->sgmv_shrink_kind == 0 && a.n_mats <= 3 && a.tc_ksplit > 0) {
+    // long segments: the shrink on tcgen05 tensor cores, tiles of 128 tokens, its own number of d_in slices
+    a.ksplit = a.tc_ksplit;
+    sgmv::TcShrinkArgs t;
+    t.pv = a.pv;
+    t.v = a.v;
+    t.ksplit = a.ksplit;
+    t.n_mats = a.n_mats;
+    for (int j = 0; j < 3; ++j) t.mat_index[j] = a.mat_index[j < a.n_mats ? j : 0];
+    t.seg_indptr = a.seg_indptr;
+    t.lora_ids = a.lora_ids;
+    t.n_seg = a.n_seg;
+    t.n_tokens = a.n_tokens;
+    t.d_in = p->mats[a.mat_index[0]].d_in;
+    const int rc = sgmv::shrink_tc(p, t, a.x, RMAX, st);
+    if (rc != FL_OK) return rc;
+  } else if (TM == 64 && RMAX == 16 && a.n_mats == 3) {      // at higher ranks the three accumulators cost too many registers
     static bool configured3[16] = {};
     const int smem3 = (RMAX == 64 ? 3 : 4) * (64 + 3 * RMAX) * 128;
     if (!configured3[p->device & 15]) {
@@ -724,10 +694,24 @@ int sgmv_common(fl_pool* p, fl_bf16* const* ys, const fl_bf16* x, const int* mat
     const size_t need = (size_t)n_mats * 2 * (size_t)n_tokens * rmax * sizeof(float) + 256;
     if (shrink_ctas < 592 && need <= workspace_bytes) a.ksplit = 2;
   }
+  a.tc_ksplit = 0;
+  if (!small && n_mats <= 3 && rmax >= 32) {     // at rank 16 the mma.sync shrink is the faster one
+    // units of (128-token tile, slice of d_in) for the tcgen05 shrink: about four per SM when the scratch the caller
+    // brought has room for the slices, every slice at least 512 values deep
+    const int d_in = p->mats[mat_indices[0]].d_in;
+    const long tiles = (long)n_seg + n_tokens / 128;
+    int ks = (int)std::min<long>(8, std::max<long>(1, (4L * p->sm_count + tiles - 1) / tiles));
+    ks = std::min(ks, std::max(1, d_in / 512));
+    // (measured against the size every caller has to bring, not against what this caller brought: the number of
+    // slices fixes the order of the sums, and equal calls should give equal bits)
+    const size_t room = fl_lora_sgmv_workspace(n_tokens, n_mats);
+    while (ks > 1 && (size_t)n_mats * ks * (size_t)n_tokens * rmax * sizeof(float) + 256 > room) --ks;
+    if ((size_t)n_mats * ks * (size_t)n_tokens * rmax * sizeof(float) + 256 <= room) a.tc_ksplit = ks;
+  }
   int rc;
   const bool so = shrink_only != nullptr;
   if (so) {
-    shrink_only->ksplit = a.ksplit;
+    shrink_only->ksplit = (!small && p->sgmv_shrink_kind == 0 && a.tc_ksplit > 0) ? a.tc_ksplit : a.ksplit;
     shrink_only->rmax = rmax;
   }
   if (small) {

@@ -19,6 +19,7 @@
 #include <cuda.h>
 #include <string.h>
 #include <algorithm>
+#include "lora_plan.cuh"
 #include "mma_utils.cuh"
 #include "pool.cuh"
 #include "sgmv.cuh"
@@ -29,14 +30,15 @@ namespace {
 
 using namespace tc;
 
+using lora_plan::BM;
+using lora_plan::ER;
+using lora_plan::EXT_CAP;
+
 constexpr int LT_THREADS = 192;
-constexpr int BM = 128, BK = 64;
+constexpr int BK = 64;
 constexpr int MAX_LIN = 3;                       // projections per launch (q, k, v share x)
 constexpr uint32_t A_BYTES = BM * BK * 2;        // x tile, K-major: 128 rows of 128 bytes
 constexpr uint32_t B_GROUP = BK * 128;           // one 64-column group of a W tile: 64 k-rows of 128 bytes
-
-constexpr int ER = 32;                           // ranks per LoRA stage
-constexpr int EXT_CAP = 2 * BM;                  // LoRA stages a tile can need: every token another adapter of rank 64
 
 template <int BN>
 struct Cfg {
@@ -76,37 +78,6 @@ struct LinMaps {
   CUtensorMap x;
   CUtensorMap w[MAX_LIN];
 };
-
-// Per 128-token tile, the LoRA stages it needs: one per 32 ranks of every overlapping segment with a registered adapter.
-__global__ void __launch_bounds__(128) lin_plan_kernel(const LinArgs a, int* __restrict__ ext_count, int* __restrict__ ext_list) {
-  pdl_wait();
-  pdl_launch_dependents();
-  const int m = blockIdx.x * 128 + threadIdx.x;
-  if (m >= a.m_tiles) return;
-  const int tok0 = m * BM, tok1 = min(a.n_tokens, tok0 + BM);
-  int lo = 0, hi = a.n_seg;          // first segment that ends behind tok0
-  while (lo < hi) {
-    const int mid = (lo + hi) >> 1;
-    if (a.seg_indptr[mid + 1] > tok0) hi = mid; else lo = mid + 1;
-  }
-  int c = 0;
-  for (int s = lo; s < a.n_seg && c + 2 <= EXT_CAP; ++s) {
-    const int s0 = a.seg_indptr[s], s1 = a.seg_indptr[s + 1];
-    if (s0 >= tok1) break;
-    if (s1 <= s0 || s1 <= tok0) continue;
-    const int lid = a.lora_ids[s];
-    if (lid < 0) continue;
-    bool ok = (uint32_t)lid < a.pv.dir_cap && a.pv.dir[lid].rank > 0;
-    for (int j = 0; ok && j < a.n_mats; ++j) ok = a.mat_index[j] < a.pv.dir[lid].n_mats;
-    if (!ok) {
-      atomicOr(a.pv.flags, (uint32_t)FLAG_BAD_LORA);
-      continue;
-    }
-    ext_list[(size_t)m * EXT_CAP + c++] = s << 1;
-    if (a.pv.dir[lid].rank > ER) ext_list[(size_t)m * EXT_CAP + c++] = s << 1 | 1;
-  }
-  ext_count[m] = c;
-}
 
 struct Tile {
   int j, m, n;       // projection, token tile, column tile
@@ -511,7 +482,16 @@ int fl_lora_linear_multi(fl_pool* p, fl_bf16* const* ys, const fl_bf16* x, const
     }
     for (int j = n_mats; j < MAX_LIN; ++j) maps.w[j] = maps.w[0];
     if (rc != FL_OK) break;
-    if (launch_pdl(lin_plan_kernel, dim3((lw.m_tiles + 127) / 128), dim3(128), 0, st, a, ext_count, ext_list) != cudaSuccess) {
+    lora_plan::PlanArgs pa;
+    pa.pv = a.pv;
+    pa.seg_indptr = a.seg_indptr;
+    pa.lora_ids = a.lora_ids;
+    pa.n_seg = a.n_seg;
+    pa.n_tokens = n_tokens;
+    pa.m_tiles = lw.m_tiles;
+    pa.n_mats = n_mats;
+    for (int j = 0; j < FL_MAX_MATS; ++j) pa.mat_index[j] = j < n_mats ? a.mat_index[j] : 0;
+    if (lora_plan::launch_plan(pa, ext_count, ext_list, st) != cudaSuccess) {
       p->last_cuda = (int)cudaGetLastError();
       rc = FL_ECUDA;
       break;

@@ -320,13 +320,11 @@ def bench_workload(args, name, world, rank, local, oracle_budget_s):
             mark()
 
     # the same layer with its base projections on the path: every projection is one GEMM that also takes the LoRA term
-    fused_calls = ["linear_qkv", "kv_append", "attention", "linear_o"] + (["linear_up", "linear_down"] if s.inter else [])
+    fused_calls = ["linear_qkv_append", "attention", "linear_o"] + (["linear_up", "linear_down"] if s.inter else [])
 
     def fused_call(c):
-        if c == "linear_qkv":
-            sess.lora_linear([d_z["q"], d_z["k"], d_z["v"]], d_x, [d_w["q"], d_w["k"], d_w["v"]], ["q", "k", "v"], stream=main)
-        elif c == "kv_append":
-            sess.kv_append(d_z["k"], d_z["v"], stream=main)
+        if c == "linear_qkv_append":      # q to d_z["q"], k and v straight into the requests' pool blocks
+            sess.lora_linear_qkv_append(d_z["q"], d_x, d_w["q"], d_w["k"], d_w["v"], stream=main)
         elif c == "attention":
             sess.attention(d_attn, d_z["q"], stream=main)
         elif c == "linear_o":
@@ -560,7 +558,7 @@ def bench_workload(args, name, world, rank, local, oracle_budget_s):
         for c in fused_calls:
             e = {"ms": round(fused_ms[c], 4)}
             if c.startswith("linear"):
-                mats = {"linear_qkv": ["q", "k", "v"], "linear_o": ["o"], "linear_up": ["up"], "linear_down": ["down"]}[c]
+                mats = {"linear_qkv_append": ["q", "k", "v"], "linear_o": ["o"], "linear_up": ["up"], "linear_down": ["down"]}[c]
                 fl_ = sum(2.0 * T * dims[m][0] * dims[m][1] for m in mats)
                 by = 2 * T * dims[mats[0]][0] + sum(2 * T * dims[m][1] + 2 * dims[m][0] * dims[m][1] for m in mats)
                 e.update({"ms_back_to_back": round(b2b_ms[c], 4), "gemm_flops": fl_,
@@ -570,8 +568,8 @@ def bench_workload(args, name, world, rank, local, oracle_budget_s):
                           "algorithmic_bytes": int(by), "frac_hbm": round(by / (fused_ms[c] * 1e-3) / 1e9 / pk["hbm"], 4),
                           "bound": "tensor" if fl_ / by > 250 else "hbm"})
             fused["calls"][c] = e
-        fused["note"] = "x W + s (x A) B per projection in one tcgen05 GEMM (y written once, no read-modify-write), " \
-                        "KV append, attention; weights resident in HBM"
+        fused["note"] = "x W + s (x A) B per projection in one tcgen05 GEMM (y written once, no read-modify-write; K and V " \
+                        "rows go from the accumulator straight into the pool blocks), attention; weights resident in HBM"
         cb, _, _ = oracle_baseline(wl, budget_s=oracle_budget_s)
         rec = {
             "value": tokens_all / (ms_step * 1e-3), "unit": "tokens/s", "ms_per_step": ms_step,

@@ -246,6 +246,21 @@ int fl_lora_linear_multi(fl_pool* pool, fl_bf16* const* ys, const fl_bf16* x, co
                          int n_seg, int n_tokens, float scale, void* workspace, size_t workspace_bytes,
                          fl_stream stream);
 
+/* The q, k, v projections of a layer from x and the base weights, with the KV store folded in (Eq. 2 and Section 4.3
+ * in one pass): q = x W_q + LoRA term goes to y_q; the k and v rows are never written anywhere but into the requests'
+ * pool blocks, at the positions and in the layout of fl_kv_append (cleared V slots behind a request's last token
+ * included).  Bit for bit what fl_lora_linear_multi followed by fl_kv_append stores.  mat_k and mat_v must have
+ * d_out = n_kv_heads * 128.  scratch_k, scratch_v: device [n_tokens, n_kv_heads * 128] bf16 each, needed only by
+ * batches of short segments (n_tokens <= 16 * n_seg, e.g. a decode step), where x W is formed first and the segmented
+ * projection then stores base + LoRA term; may be NULL otherwise (FL_EINVAL if such a batch comes without them).
+ * workspace as fl_lora_linear_workspace(n_tokens, 3). */
+int fl_lora_linear_qkv_append(fl_pool* pool, fl_bf16* y_q, const fl_bf16* x, const fl_bf16* w_q, const fl_bf16* w_k,
+                              const fl_bf16* w_v, int mat_q, int mat_k, int mat_v, const int32_t* seg_indptr,
+                              const int32_t* lora_ids, int n_seg, int n_tokens, float scale, const int32_t* req_indptr,
+                              const int32_t* kv_tbl_indptr, const uint32_t* kv_tbl, const int32_t* prefix_lens, int n_req,
+                              int n_kv_heads, fl_bf16* scratch_k, fl_bf16* scratch_v, void* workspace,
+                              size_t workspace_bytes, fl_stream stream);
+
 /* ---------------------------------------------------------------- KV store (Section 4.3: new KV stays in HBM blocks)
  * Writes the new tokens' K and V into the pool.  Request i owns tokens req_indptr[i] .. req_indptr[i+1]
  * of k_new / v_new (device, [n_tokens, n_kv_heads, 128] bf16); its token j goes to logical position

@@ -105,6 +105,9 @@ _SIGS = {
     "fl_lora_linear": (C.c_int, [_vp, _vp, _vp, _vp, C.c_int, _vp, _vp, C.c_int, C.c_int, C.c_float, _vp, C.c_size_t, _vp]),
     "fl_lora_linear_multi": (C.c_int, [_vp, C.POINTER(_vp), _vp, C.POINTER(_vp), _i32p, C.c_int, _vp, _vp, C.c_int,
                                        C.c_int, C.c_float, _vp, C.c_size_t, _vp]),
+    "fl_lora_linear_qkv_append": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, C.c_int, C.c_int, C.c_int, _vp, _vp, C.c_int,
+                                            C.c_int, C.c_float, _vp, _vp, _vp, _vp, C.c_int, C.c_int, _vp, _vp, _vp,
+                                            C.c_size_t, _vp]),
     "fl_kv_append": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, C.c_int, C.c_int, C.c_int, _vp]),
     "fl_paged_attention_workspace": (C.c_size_t, [C.c_int, C.c_int, C.c_int, C.c_int, C.c_int]),
     "fl_paged_attention": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, C.c_int, C.c_int, C.c_int, C.c_int,
@@ -349,6 +352,17 @@ def fl_lora_linear_multi(pool, ys, x, ws, mat_indices, seg_indptr, lora_ids, n_s
     _check(lib.fl_lora_linear_multi(pool, py, _dev(x), pw, mi, len(ys), _dev(seg_indptr), _dev(lora_ids), n_seg,
                                     n_tokens, scale, _dev(workspace), workspace.numel() * workspace.element_size(),
                                     _stream(stream)), "fl_lora_linear_multi")
+
+
+def fl_lora_linear_qkv_append(pool, y_q, x, w_q, w_k, w_v, mat_q, mat_k, mat_v, seg_indptr, lora_ids, n_seg, n_tokens,
+                              scale, req_indptr, kv_tbl_indptr, kv_tbl, prefix_lens, n_req, n_kv_heads, scratch_k,
+                              scratch_v, workspace, stream=None):
+    _check(lib.fl_lora_linear_qkv_append(pool, _dev(y_q), _dev(x), _dev(w_q), _dev(w_k), _dev(w_v), mat_q, mat_k, mat_v,
+                                         _dev(seg_indptr), _dev(lora_ids), n_seg, n_tokens, scale, _dev(req_indptr),
+                                         _dev(kv_tbl_indptr), _dev(kv_tbl), _dev(prefix_lens), n_req, n_kv_heads,
+                                         _dev(scratch_k), _dev(scratch_v), _dev(workspace),
+                                         workspace.numel() * workspace.element_size(), _stream(stream)),
+           "fl_lora_linear_qkv_append")
 
 
 def fl_kv_append(pool, k_new, v_new, req_indptr, kv_tbl_indptr, kv_tbl, prefix_lens, n_req, n_tokens, n_kv_heads,

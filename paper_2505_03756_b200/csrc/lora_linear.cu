@@ -72,6 +72,13 @@ struct LinArgs {
   int m_tiles;
   const int* ext_count;        // per 128-token tile: LoRA stages (32 ranks of one overlapping segment's adapter)
   const int* ext_list;         // [m_tiles][EXT_CAP]: segment << 1 | which half of the ranks
+  // K / V projections whose rows go straight into the requests' pool blocks (kv_side: -1 = rows go to y, 0 = K, 1 = V)
+  int kv_side[MAX_LIN];
+  const int32_t* req_indptr;
+  const int32_t* tbl_indptr;
+  const uint32_t* tbl;
+  const int32_t* prefix_lens;
+  int n_req, n_kv, bt;
 };
 
 struct LinMaps {
@@ -316,13 +323,39 @@ __global__ void __launch_bounds__(LT_THREADS, 1) lora_linear_kernel(const LinArg
       if (idx + (int)gridDim.x < total) fill_ext(idx + gridDim.x);
       if (!ok) break;
       const int buf = k & 1;
-      ok = group_and(mbar_wait(bar(B_ACC_FULL + buf), (uint32_t)((k >> 1) & 1), abort_flag), 1, 128);
-      if (!ok) break;
-      tc_fence_after();
       const int tok = t.m * BM + row;
       const int d_out = a.d_out[t.j];
       const int n0 = t.n * BN;
-      __nv_bfloat16* yrow = a.y[t.j] + (size_t)tok * d_out + n0;
+      const int side = a.kv_side[t.j];
+      // a K / V row belongs in its token's pool block: block and slot of the token's position, found while the
+      // tile's MMAs are still running
+      uint32_t kv_blk = 0;
+      int kv_slot = -1, kv_last = 0;
+      if (side >= 0 && tok < a.n_tokens) {
+        int lo = 0, hi = a.n_req;
+        while (hi - lo > 1) {
+          const int mid = (lo + hi) >> 1;
+          if (a.req_indptr[mid] <= tok) lo = mid; else hi = mid;
+        }
+        const int pos = a.prefix_lens[lo] + (tok - a.req_indptr[lo]);
+        const int entry = pos / a.bt, slot = pos - entry * a.bt;
+        if (pos < 0 || tok < a.req_indptr[lo] || tok >= a.req_indptr[lo + 1] || entry >= a.tbl_indptr[lo + 1] - a.tbl_indptr[lo]) {
+          atomicOr(a.pv.flags, (uint32_t)FLAG_BAD_POS);
+        } else {
+          const uint32_t blk = a.tbl[a.tbl_indptr[lo] + entry];
+          if (blk >= a.pv.n_blocks) {
+            atomicOr(a.pv.flags, (uint32_t)FLAG_BAD_BLOCK);
+          } else {
+            kv_blk = blk;
+            kv_slot = slot;
+            kv_last = tok == a.req_indptr[lo + 1] - 1;
+          }
+        }
+      }
+      ok = group_and(mbar_wait(bar(B_ACC_FULL + buf), (uint32_t)((k >> 1) & 1), abort_flag), 1, 128);
+      if (!ok) break;
+      tc_fence_after();
+      __nv_bfloat16* yrow = side < 0 ? a.y[t.j] + (size_t)tok * d_out + n0 : nullptr;
 #pragma unroll 2
       for (int cb = 0; cb < BN; cb += 32) {
         uint32_t o[32];
@@ -337,7 +370,19 @@ __global__ void __launch_bounds__(LT_THREADS, 1) lora_linear_kernel(const LinArg
               q.y = pack_bf16(__uint_as_float(o[8 * c + 2]), __uint_as_float(o[8 * c + 3]));
               q.z = pack_bf16(__uint_as_float(o[8 * c + 4]), __uint_as_float(o[8 * c + 5]));
               q.w = pack_bf16(__uint_as_float(o[8 * c + 6]), __uint_as_float(o[8 * c + 7]));
-              *reinterpret_cast<uint4*>(yrow + cb + 8 * c) = q;
+              if (side < 0) {
+                *reinterpret_cast<uint4*>(yrow + cb + 8 * c) = q;
+              } else if (kv_slot >= 0) {
+                // [K|V][kv head][slot][128] inside the block
+                const int colg = n0 + cb + 8 * c;
+                unsigned char* dst = a.pv.slab + (size_t)kv_blk * a.pv.block_bytes +
+                                     ((size_t)(side * a.n_kv + colg / FL_HEAD_DIM) * a.bt + kv_slot) * (FL_HEAD_DIM * 2) +
+                                     (colg % FL_HEAD_DIM) * 2;
+                *reinterpret_cast<uint4*>(dst) = q;
+                if (side == 1 && kv_last)       // V of a request's last token: clear the slots behind it
+                  for (int z = kv_slot + 1; z < a.bt; ++z)
+                    *reinterpret_cast<uint4*>(dst + (z - kv_slot) * (FL_HEAD_DIM * 2)) = make_uint4(0u, 0u, 0u, 0u);
+              }
             }
           }
         }
@@ -407,10 +452,27 @@ size_t fl_lora_linear_workspace(int n_tokens, int n_mats) {
   return lin_ws(n_tokens, n_mats).total;
 }
 
-int fl_lora_linear_multi(fl_pool* p, fl_bf16* const* ys, const fl_bf16* x, const fl_bf16* const* ws, const int* mat_indices,
-                         int n_mats, const int32_t* seg_indptr, const int32_t* lora_ids, int n_seg, int n_tokens,
-                         float scale, void* workspace, size_t workspace_bytes, fl_stream stream) {
-  if (!p || n_mats < 1 || n_mats > MAX_LIN || n_seg < 0 || n_tokens < 0 || !ys || !ws || !mat_indices) return FL_EINVAL;
+}  // extern "C"
+
+namespace {
+
+struct LinKv {        // K and V projections of the call whose rows go into pool blocks
+  int k_slot, v_slot;
+  const int32_t* req_indptr;
+  const int32_t* tbl_indptr;
+  const uint32_t* tbl;
+  const int32_t* prefix_lens;
+  int n_req, n_kv;
+  fl_bf16* tmp_k;     // [n_tokens, n_kv * 128] each: needed by batches of short segments only
+  fl_bf16* tmp_v;
+};
+
+int linear_common(fl_pool* p, fl_bf16* const* ys_in, const fl_bf16* x, const fl_bf16* const* ws, const int* mat_indices,
+                  int n_mats, const int32_t* seg_indptr, const int32_t* lora_ids, int n_seg, int n_tokens,
+                  float scale, void* workspace, size_t workspace_bytes, fl_stream stream, const LinKv* kv) {
+  if (!p || n_mats < 1 || n_mats > MAX_LIN || n_seg < 0 || n_tokens < 0 || !ys_in || !ws || !mat_indices) return FL_EINVAL;
+  fl_bf16* ys[MAX_LIN] = {};
+  for (int j = 0; j < n_mats; ++j) ys[j] = ys_in[j];
   if (n_tokens == 0) return FL_OK;
   if (!x || !workspace || (n_seg > 0 && (!seg_indptr || !lora_ids))) return FL_EINVAL;
   if (p->n_mats == 0) return FL_EBADID;           // the projection shapes come with the first registered adapter
@@ -422,7 +484,8 @@ int fl_lora_linear_multi(fl_pool* p, fl_bf16* const* ys, const fl_bf16* x, const
   int d_out_min = 1 << 30;
   for (int j = 0; j < n_mats; ++j) {
     const int mi = mat_indices[j];
-    if (mi < 0 || mi >= p->n_mats || !ys[j] || !ws[j]) return FL_EINVAL;
+    const bool to_pool = kv && (j == kv->k_slot || j == kv->v_slot);
+    if (mi < 0 || mi >= p->n_mats || (!ys[j] && !to_pool) || !ws[j]) return FL_EINVAL;
     if (p->mats[mi].d_in != p->mats[mat_indices[0]].d_in) return FL_EINVAL;   // the projections share x
     a.y[j] = reinterpret_cast<__nv_bfloat16*>(ys[j]);
     a.mat_index[j] = mi;
@@ -448,6 +511,31 @@ int fl_lora_linear_multi(fl_pool* p, fl_bf16* const* ys, const fl_bf16* x, const
   // and the segmented projection adds the LoRA term to y afterwards.
   const bool hybrid = n_seg > 0 && n_tokens <= 16 * n_seg;
   if (hybrid) a.n_seg = 0;
+  for (int j = 0; j < MAX_LIN; ++j) a.kv_side[j] = -1;
+  if (kv) {
+    const size_t per_tok = (size_t)2 * kv->n_kv * FL_HEAD_DIM * 2;
+    if (kv->n_kv < 1 || kv->n_req < 1 || p->block_bytes % per_tok != 0 || kv->k_slot == kv->v_slot) return FL_EINVAL;
+    if (!kv->req_indptr || !kv->tbl_indptr || !kv->tbl || !kv->prefix_lens) return FL_EINVAL;
+    for (int side = 0; side < 2; ++side) {
+      const int slot = side ? kv->v_slot : kv->k_slot;
+      if (slot < 0 || slot >= n_mats || a.d_out[slot] != kv->n_kv * FL_HEAD_DIM) return FL_EINVAL;
+      if (hybrid) {      // x W goes to a scratch row first; the segmented projection then stores base + LoRA term in the pool
+        fl_bf16* tmp = side ? kv->tmp_v : kv->tmp_k;
+        if (!tmp) return FL_EINVAL;
+        ys[slot] = tmp;
+        a.y[slot] = reinterpret_cast<__nv_bfloat16*>(tmp);
+      } else {
+        a.kv_side[slot] = side;
+      }
+    }
+    a.req_indptr = kv->req_indptr;
+    a.tbl_indptr = kv->tbl_indptr;
+    a.tbl = kv->tbl;
+    a.prefix_lens = kv->prefix_lens;
+    a.n_req = kv->n_req;
+    a.n_kv = kv->n_kv;
+    a.bt = (int)(p->block_bytes / per_tok);
+  }
   // few token tiles: narrower column tiles, so that every SM streams a slice of W
   int bn = 256;
   {
@@ -504,8 +592,16 @@ int fl_lora_linear_multi(fl_pool* p, fl_bf16* const* ys, const fl_bf16* x, const
       rc = info.rmax == 16 ? launch_linear<64, 16>(p, a, maps, st) : info.rmax == 32 ? launch_linear<64, 32>(p, a, maps, st)
                                                                                    : launch_linear<64, 64>(p, a, maps, st);
       if (rc != FL_OK) break;
-      rc = fl_lora_sgmv_multi(p, ys, x, mat_indices, n_mats, seg_indptr, lora_ids, n_seg, n_tokens, scale, wsb + lw.v,
-                              fl_lora_sgmv_workspace(n_tokens, n_mats), stream);
+      if (kv && n_mats == 3 && kv->k_slot == 1 && kv->v_slot == 2)
+        rc = fl_lora_sgmv_qkv_append(p, ys[0], ys[1], ys[2], x, mat_indices[0], mat_indices[1], mat_indices[2], seg_indptr,
+                                     lora_ids, n_seg, n_tokens, scale, kv->req_indptr, kv->tbl_indptr, kv->tbl,
+                                     kv->prefix_lens, kv->n_req, kv->n_kv, wsb + lw.v,
+                                     fl_lora_sgmv_workspace(n_tokens, n_mats), stream);
+      else if (kv)
+        rc = FL_EINVAL;
+      else
+        rc = fl_lora_sgmv_multi(p, ys, x, mat_indices, n_mats, seg_indptr, lora_ids, n_seg, n_tokens, scale, wsb + lw.v,
+                                fl_lora_sgmv_workspace(n_tokens, n_mats), stream);
       break;
     }
     if (n_seg > 0) {
@@ -524,6 +620,31 @@ int fl_lora_linear_multi(fl_pool* p, fl_bf16* const* ys, const fl_bf16* x, const
   } while (0);
   if (prev != p->device && prev >= 0) cudaSetDevice(prev);
   return rc;
+}
+
+}  // namespace
+
+extern "C" {
+
+int fl_lora_linear_multi(fl_pool* p, fl_bf16* const* ys, const fl_bf16* x, const fl_bf16* const* ws, const int* mat_indices,
+                         int n_mats, const int32_t* seg_indptr, const int32_t* lora_ids, int n_seg, int n_tokens,
+                         float scale, void* workspace, size_t workspace_bytes, fl_stream stream) {
+  return linear_common(p, ys, x, ws, mat_indices, n_mats, seg_indptr, lora_ids, n_seg, n_tokens, scale, workspace,
+                       workspace_bytes, stream, nullptr);
+}
+
+int fl_lora_linear_qkv_append(fl_pool* p, fl_bf16* y_q, const fl_bf16* x, const fl_bf16* w_q, const fl_bf16* w_k,
+                              const fl_bf16* w_v, int mat_q, int mat_k, int mat_v, const int32_t* seg_indptr,
+                              const int32_t* lora_ids, int n_seg, int n_tokens, float scale, const int32_t* req_indptr,
+                              const int32_t* kv_tbl_indptr, const uint32_t* kv_tbl, const int32_t* prefix_lens, int n_req,
+                              int n_kv_heads, fl_bf16* scratch_k, fl_bf16* scratch_v, void* workspace,
+                              size_t workspace_bytes, fl_stream stream) {
+  fl_bf16* ys[3] = {y_q, nullptr, nullptr};
+  const fl_bf16* ws[3] = {w_q, w_k, w_v};
+  const int mi[3] = {mat_q, mat_k, mat_v};
+  const LinKv kv = {1, 2, req_indptr, kv_tbl_indptr, kv_tbl, prefix_lens, n_req, n_kv_heads, scratch_k, scratch_v};
+  return linear_common(p, ys, x, ws, mi, 3, seg_indptr, lora_ids, n_seg, n_tokens, scale, workspace, workspace_bytes,
+                       stream, &kv);
 }
 
 int fl_lora_linear(fl_pool* p, fl_bf16* y, const fl_bf16* x, const fl_bf16* w, int mat_index,

@@ -186,6 +186,21 @@ class Session:
         fl.fl_lora_linear_multi(self.pool, ys, x, ws, [self.mat_index[m] for m in mats], self.t_seg_indptr,
                                 self.t_seg_lora, self.n_seg, T, scale, wsp, stream)
 
+    def lora_linear_qkv_append(self, y_q, x, w_q, w_k, w_v, scale=None, stream=None):
+        """q = x W_q + LoRA term into y_q; k, v = x W + LoRA term straight into the batch's pool blocks."""
+        T, s = self.wl.n_tokens, self.shape
+        wsp = self.workspace("linear", fl.fl_lora_linear_workspace(T, 3))
+        scale = self.wl.scale if scale is None else scale
+        tmp_k = tmp_v = None
+        if T <= 16 * self.n_seg:           # short segments: the library forms x W in scratch rows first
+            tmp = self.workspace("linear_kv", 2 * T * s.n_kv_heads * s.head_dim * 2)
+            half = T * s.n_kv_heads * s.head_dim * 2
+            tmp_k, tmp_v = tmp[:half], tmp[half:2 * half]
+        fl.fl_lora_linear_qkv_append(self.pool, y_q, x, w_q, w_k, w_v, self.mat_index["q"], self.mat_index["k"],
+                                     self.mat_index["v"], self.t_seg_indptr, self.t_seg_lora, self.n_seg, T, scale,
+                                     self.t_req_indptr, self.t_tbl_indptr, self.t_tbl, self.t_prefix, self.wl.n_req,
+                                     s.n_kv_heads, tmp_k, tmp_v, wsp, stream)
+
     def sgmv_qkv_append(self, y_q, y_k, y_v, x, scale=None, stream=None):
         """q += LoRA term in place; base k, v + LoRA term written straight into the batch's pool blocks."""
         T = self.wl.n_tokens

@@ -1,7 +1,9 @@
 """The four large workloads at their full sizes, run as bench.py runs them (one layer step through the
-C ABI), checked against the CPU oracle on sampled outputs: token rows of every LoRA projection, appended
-KV rows bit for bit, attention rows (first and last new token of sampled requests plus random rows), and
-the allocator trace.  Every sampled output is computed by the oracle from the stage's own inputs."""
+C ABI: the q/k/v projection with the KV store folded in, attention, the o projection), checked against the CPU
+oracle on sampled outputs: token rows of every LoRA projection (K and V rows read back out of their pool blocks),
+attention rows (first and last new token of sampled requests plus random rows), and the allocator trace.  Every
+sampled output is computed by the oracle from the stage's own inputs.  A second test does the same for the layer
+with its base projections on the path (fl_lora_linear)."""
 import math
 
 import numpy as np
@@ -11,7 +13,7 @@ torch = pytest.importorskip("torch")
 pytestmark = pytest.mark.gpu
 
 from oracle.attention import attend_rows
-from oracle.lora import lora_project
+from oracle.lora import lora_linear, lora_project
 from paper_2505_03756_b200 import synth
 
 from _util import assert_close, replay_trace
@@ -76,8 +78,7 @@ def test_full_size_layer_step_sampled(name):
             yb_rows[m] = yb[rows].astype(np.float64)
             ty[m] = H.f32_to_dev(yb, s.dev)
             del yb
-        s.sgmv([ty["q"], ty["k"], ty["v"]], tx, ["q", "k", "v"])
-        s.kv_append(ty["k"], ty["v"])
+        s.sgmv_qkv_append(ty["q"], ty["k"], ty["v"], tx)          # k, v results go to the pool blocks only
         attn = torch.empty(T, sh.n_q_heads, 128, dtype=torch.bfloat16, device=s.dev)
         s.attention(attn, ty["q"])
         yb = wl.y_base("o")
@@ -92,10 +93,32 @@ def test_full_size_layer_step_sampled(name):
         def take(t):
             return H.dev_to_f32(t.view(T, -1)[trows]).astype(np.float64)
 
-        # a2/a3: sampled rows of every projection
+        bt = sh.block_tokens
+        blocks = {}
+
+        def block(b):
+            if b not in blocks:
+                blocks[b] = fl.fl_block_read(s.pool, int(b), s.block_bytes).view(np.uint16).reshape(2, sh.n_kv_heads, bt, 128)
+            return blocks[b]
+
+        def kv_rows_from_pool(tokens):
+            """K and V rows of the given token rows, read through the requests' block tables: [n, 2, n_kv * 128]."""
+            out = np.empty((len(tokens), 2, sh.n_kv_heads * 128), dtype=np.float64)
+            for k, t in enumerate(tokens):
+                i = int(np.searchsorted(wl.req_indptr, t, side="right") - 1)
+                pos = int(wl.prefix_lens[i]) + int(t) - int(wl.req_indptr[i])
+                blk = block(s.kv_tables[i][pos // bt])
+                out[k] = synth.bf16_to_f32(blk[:, :, pos % bt, :]).reshape(2, -1)
+            return out
+
+        # a2/a3 (+ a4): sampled rows of every projection; k and v come out of the pool blocks
         x_rows = x[rows].astype(np.float64)
-        for m in "qkv":
-            _check_projection(H, wl, rows, x_rows, yb_rows[m], take(ty[m]), m, f"{name}/{m}")
+        kv_got = kv_rows_from_pool(rows)
+        _check_projection(H, wl, rows, x_rows, yb_rows["q"], take(ty["q"]), "q", f"{name}/q")
+        _check_projection(H, wl, rows, x_rows, yb_rows["k"], kv_got[:, 0], "k", f"{name}/k in pool")
+        _check_projection(H, wl, rows, x_rows, yb_rows["v"], kv_got[:, 1], "v", f"{name}/v in pool")
+        for m in "kv":      # the inputs of the fused call are left as they were
+            assert np.array_equal(take(ty[m]), yb_rows[m]), m
         _check_projection(H, wl, rows, take(attn), yb_rows["o"], take(ty["o"]), "o", f"{name}/o")
         if sh.inter:
             for m, src in (("up", "o"), ("down", "up")):
@@ -110,23 +133,20 @@ def test_full_size_layer_step_sampled(name):
         # a1: allocator trace replayed on the model, free lists bit for bit
         model = replay_trace(s)
         assert np.array_equal(fl.fl_pool_snapshot(s.pool), np.array(model.free_list(), dtype=np.uint32))
-        # a4 + a5/a6 on sampled requests
-        bt = sh.block_tokens
+        # a5/a6 on sampled requests: the context is the cached prefix plus the new K, V as the pool holds them
         reqs = sorted(set(int(r) for r in rs.integers(0, wl.n_req - 1, N_REQ)) | {0, wl.n_req - 1})
-        k_all, v_all, q_all = ty["k"].view(T, sh.n_kv_heads, 128), ty["v"].view(T, sh.n_kv_heads, 128), ty["q"].view(T, sh.n_q_heads, 128)
+        q_all = ty["q"].view(T, sh.n_q_heads, 128)
         for i in reqs:
             lo, hi = int(wl.req_indptr[i]), int(wl.req_indptr[i + 1])
             n, p = hi - lo, int(wl.prefix_lens[i])
             if n == 0:
                 continue
-            k_new, v_new = H.dev_to_f32(k_all[lo:hi]), H.dev_to_f32(v_all[lo:hi])
-            # KV rows of the first and last new token, bit for bit, read back from their pool blocks
-            for j in {0, n - 1}:
-                pos = p + j
-                blk = fl.fl_block_read(s.pool, int(s.kv_tables[i][pos // bt]), s.block_bytes).view(np.uint16)
-                blk = blk.reshape(2, sh.n_kv_heads, bt, 128)
-                assert np.array_equal(blk[0, :, pos % bt], synth.bf16_bits(k_new[j])), (name, i, j)
-                assert np.array_equal(blk[1, :, pos % bt], synth.bf16_bits(v_new[j])), (name, i, j)
+            kv_new = kv_rows_from_pool(np.arange(lo, hi)).reshape(n, 2, sh.n_kv_heads, 128)
+            k_new, v_new = kv_new[:, 0], kv_new[:, 1]
+            # V slots behind the request's last token are cleared
+            last = p + n - 1
+            if (last + 1) % bt:
+                assert not block(s.kv_tables[i][last // bt])[1, :, last % bt + 1:, :].any(), (name, i)
             kp, vp = wl.kv_prefix(i)
             k_ctx = np.concatenate([kp, k_new]).astype(np.float64)
             v_ctx = np.concatenate([vp, v_new]).astype(np.float64)
@@ -135,5 +155,49 @@ def test_full_size_layer_step_sampled(name):
             want = attend_rows(q_rows, [p + j for j in js], k_ctx, v_ctx, 1.0 / math.sqrt(128))
             got = H.dev_to_f32(attn[lo:hi][js])
             assert_close(got, want, f"{name}/attention request {i}")
+    finally:
+        s.close()
+
+
+@pytest.mark.parametrize("name", ["prefill7b", "decode13b", "gqa34b", "swapstress"])
+def test_full_size_fused_projections_sampled(name):
+    """y = x W + s (x A) B in one GEMM (fl_lora_linear) at the full batch sizes, sampled token rows against the oracle."""
+    assert torch.cuda.is_available(), "these tests need a GPU"
+    from paper_2505_03756_b200 import harness as H
+    wl = synth.make_workload(name)
+    if name == "gqa34b":                    # the same batch in a pool that just fits (the 60 GB slab adds nothing here)
+        wl.pool_blocks = int(sum(-(-(int(p) + int(n)) // wl.shape.block_tokens) for p, n in zip(wl.prefix_lens, wl.new_lens))) + 2000
+    sh, T = wl.shape, wl.n_tokens
+    s = H.Session(wl, scramble=False, register_all=(name == "swapstress"))
+    try:
+        s.load_adapters()
+        s.build_batch()
+        rs = synth.Stream(wl.seed, "fullsize-linear")
+        rows = _rows_sample(wl, rs)
+        lids = _seg_of_rows(wl, rows)
+        trows = torch.from_numpy(rows).to(s.dev)
+        dims = {n: (i, o) for n, i, o in sh.mats}
+        groups = [["q", "k", "v"], ["o"]] + ([["up"], ["down"]] if sh.inter else [])
+        for grp in groups:
+            x = wl.x(grp[0])
+            tx = H.f32_to_dev(x, s.dev)
+            tw = [H.f32_to_dev(wl.weight(m), s.dev) for m in grp]
+            ty = [torch.empty(T, dims[m][1], dtype=torch.bfloat16, device=s.dev) for m in grp]
+            s.lora_linear(ty, tx, tw, grp)
+            torch.cuda.synchronize()
+            assert s.status()["device_flags"] == 0
+            x_rows = x[rows].astype(np.float64)
+            for m, t in zip(grp, ty):
+                W = wl.weight(m)
+                want = np.empty((len(rows), dims[m][1]), dtype=np.float64)
+                for r in range(len(rows)):
+                    ad = {int(lids[r]): wl.adapter(int(lids[r]), m)}
+                    want[r] = lora_linear(x_rows[r:r + 1], W, [0, 1], [int(lids[r])], ad, wl.scale)[0]
+                got = H.dev_to_f32(t[trows]).astype(np.float64)
+                assert_close(got, want, f"{name}/linear {m}")
+                base = x_rows @ W.astype(np.float64)
+                rms = lambda a: float(np.sqrt(np.mean(a * a)))
+                assert rms((got - base) - (want - base)) <= 2.0 ** -8 * rms(want), (name, m, "LoRA term")
+            del tx, tw, ty
     finally:
         s.close()

@@ -6,10 +6,11 @@ import pytest
 torch = pytest.importorskip("torch")
 pytestmark = pytest.mark.gpu
 
+from oracle import pool as op
 from oracle.lora import lora_linear
 from paper_2505_03756_b200 import synth
 
-from _util import REDUCED, assert_close, oracle_adapters
+from _util import REDUCED, assert_close, oracle_adapters, replay_trace
 
 
 @pytest.fixture(scope="module")
@@ -126,5 +127,53 @@ def test_lora_linear_odd_shapes_and_ranks(H, hidden, heads, rank):
                 want = lora_linear(x, wl.weight(m), seg, ids, oracle_adapters(wl, m), wl.scale)
                 assert_close(H.dev_to_f32(t), want, f"linear {hidden}/{rank}/{m}")
         assert s.status()["device_flags"] == 0
+    finally:
+        s.close()
+
+
+@pytest.mark.parametrize("name", list(REDUCED))
+def test_lora_linear_qkv_append_stores_kv_in_the_pool(H, name):
+    """The fused q/k/v projection with the KV store folded in: q against the oracle, the pool bytes against the oracle's
+    byte model fed with the oracle's K, V, and bit for bit against projection followed by fl_kv_append."""
+    from paper_2505_03756_b200 import binding as fl
+    wl = synth.make_workload(name, **REDUCED[name])
+    s = _session(H, wl)
+    try:
+        s.fill_prefix_kv()
+        sh, T = wl.shape, wl.n_tokens
+        x = wl.x("q")
+        tx = H.f32_to_dev(x, s.dev)
+        tw = {m: H.f32_to_dev(wl.weight(m), s.dev) for m in "qkv"}
+        dims = dict((n, o) for n, _, o in sh.mats)
+        seg, ids = wl.segments()
+        tables = [[int(b) for b in t] for t in s.kv_tables]
+        blocks = sorted({b for t in tables for b in t})
+        # reference: projection into y, then the KV store
+        ty = [torch.empty(T, dims[m], dtype=torch.bfloat16, device=s.dev) for m in "qkv"]
+        s.lora_linear(ty, tx, [tw[m] for m in "qkv"], ["q", "k", "v"])
+        s.kv_append(ty[1], ty[2])
+        torch.cuda.synchronize()
+        want_blocks = fl.device_block_bytes(s.pool, s.block_bytes, blocks)
+        junk = torch.full_like(ty[1], 7.0)
+        s.kv_append(junk, junk)                      # a missing write would show
+        y_q = torch.full_like(ty[0], -5.0)
+        s.lora_linear_qkv_append(y_q, tx, tw["q"], tw["k"], tw["v"])
+        torch.cuda.synchronize()
+        assert s.status()["device_flags"] == 0
+        assert torch.equal(y_q, ty[0])
+        got_blocks = fl.device_block_bytes(s.pool, s.block_bytes, blocks)
+        assert np.array_equal(got_blocks, want_blocks), name
+        # against the oracle
+        want = {m: lora_linear(x, wl.weight(m), seg, ids, oracle_adapters(wl, m), wl.scale) for m in "qkv"}
+        assert_close(H.dev_to_f32(y_q), want["q"], f"{name}/linear+append q")
+        pos_of = {b: k for k, b in enumerate(blocks)}
+        gb = got_blocks.view(np.uint16).reshape(len(blocks), 2, sh.n_kv_heads, sh.block_tokens, 128)
+        for i in range(wl.n_req):
+            lo, hi = int(wl.req_indptr[i]), int(wl.req_indptr[i + 1])
+            pos = int(wl.prefix_lens[i]) + np.arange(hi - lo)
+            blk = np.array([pos_of[tables[i][e]] for e in pos // sh.block_tokens], dtype=np.int64)
+            rows = op.bf16_bits_to_f64(gb[blk, :, :, pos % sh.block_tokens, :])
+            assert_close(rows[:, 0].reshape(hi - lo, -1), want["k"][lo:hi], f"{name}/linear+append K in pool")
+            assert_close(rows[:, 1].reshape(hi - lo, -1), want["v"][lo:hi], f"{name}/linear+append V in pool")
     finally:
         s.close()

@@ -156,7 +156,7 @@ attn_prefill_tc2_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap kv
     asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
     if (warp == 8) {
       // ------------------------------------------------ unit fetch + TMA producer
-      // The whole warp runs the loop; lane 0 fetches units and does the waiting, lanes 0-7 each own one of a
+      // The whole warp runs the loop; lane 0 fetches units and does the waiting, lanes 0-15 each own one half of one of a
       // tile's eight pages (their block-id loads and their TMA issues run side by side).
       int fill = 0;                    // ring fills so far, over all units
       int n_valid = 0;                 // units whose Q tiles were loaded so far
@@ -197,9 +197,10 @@ attn_prefill_tc2_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap kv
         for (int j = 0; ok && j < n_kt_max; ++j) {
           // this lane's page of the tile (pages behind the last needed key are masked anyway: re-read the last
           // valid page); K_j and V_j come from the same blocks
+          // lane = 2 * page + half: sixteen lanes issue one box each
           uint32_t blk = 0;
-          if (lane < KT2 / BT) {
-            blk = a.tbl[tbl0 + min(j * (KT2 / BT) + lane, n_pages - 1)];
+          if (lane < 2 * (KT2 / BT)) {
+            blk = a.tbl[tbl0 + min(j * (KT2 / BT) + (lane >> 1), n_pages - 1)];
             if (blk >= a.pv.n_blocks) {
               atomicOr(a.pv.flags, (uint32_t)FLAG_BAD_BLOCK);
               blk = 0;
@@ -214,11 +215,10 @@ attn_prefill_tc2_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap kv
             }
             ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;     // the transaction count is armed before any copy is issued
             if (!ok) break;
-            if (lane < KT2 / BT) {
-              const uint32_t dst = sbase + OFF_RING + s * TILE_BYTES + lane * (BT * 128);
-              const int slot_head = side * a.n_kv + h;
-              tma_load_4d(dst, &kv_map, bar(C_FULL + s), 0, 0, slot_head, (int)blk);
-              tma_load_4d(dst + HALF_BYTES, &kv_map, bar(C_FULL + s), 64, 0, slot_head, (int)blk);
+            if (lane < 2 * (KT2 / BT)) {
+              const int page = lane >> 1, half = lane & 1;
+              const uint32_t dst = sbase + OFF_RING + s * TILE_BYTES + half * HALF_BYTES + page * (BT * 128);
+              tma_load_4d(dst, &kv_map, bar(C_FULL + s), 64 * half, 0, side * a.n_kv + h, (int)blk);
             }
           }
         }

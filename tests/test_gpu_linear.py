@@ -177,3 +177,40 @@ def test_lora_linear_qkv_append_stores_kv_in_the_pool(H, name):
             assert_close(rows[:, 1].reshape(hi - lo, -1), want["v"][lo:hi], f"{name}/linear+append V in pool")
     finally:
         s.close()
+
+
+def test_fused_layer_replayed_from_cuda_graph_is_bit_identical(H):
+    """The layer with its base projections, recorded once into a CUDA graph after one ordinary pass, replays bit for bit."""
+    wl = synth.make_workload("prefill7b", n_req=5, len_range=(60, 300), n_adapters=4)
+    s = _session(H, wl)
+    try:
+        s.fill_prefix_kv()
+        sh, T = wl.shape, wl.n_tokens
+        tx = H.f32_to_dev(wl.x("q"), s.dev)
+        tw = {m: H.f32_to_dev(wl.weight(m), s.dev) for m in "qkvo"}
+        y_q = torch.zeros(T, sh.n_q_heads * 128, dtype=torch.bfloat16, device=s.dev)
+        y_o = torch.zeros(T, sh.hidden, dtype=torch.bfloat16, device=s.dev)
+        attn = torch.zeros(T, sh.n_q_heads, 128, dtype=torch.bfloat16, device=s.dev)
+        main = torch.cuda.Stream()
+
+        def compute():
+            s.lora_linear_qkv_append(y_q, tx, tw["q"], tw["k"], tw["v"], stream=main)
+            s.attention(attn, y_q.view(T, sh.n_q_heads, 128), stream=main)
+            s.lora_linear([y_o], attn.view(T, -1), [tw["o"]], ["o"], stream=main)
+
+        with torch.cuda.stream(main):
+            compute()
+            main.synchronize()
+            want = (y_q.clone(), attn.clone(), y_o.clone())
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=main):
+                compute()
+            for _ in range(2):
+                for t in (y_q, attn, y_o):
+                    t.zero_()
+                g.replay()
+                main.synchronize()
+                assert torch.equal(y_q, want[0]) and torch.equal(attn, want[1]) and torch.equal(y_o, want[2])
+        assert s.status()["device_flags"] == 0
+    finally:
+        s.close()

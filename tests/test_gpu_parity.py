@@ -97,11 +97,14 @@ def test_allocator_error_paths(H):
 
 
 # ------------------------------------------------------------------ a2/a3: LoRA projection
-@pytest.mark.parametrize("name", list(REDUCED))
-def test_sgmv_parity(H, name):
+@pytest.mark.parametrize("name,shrink", [(n, 0) for n in REDUCED] + [("gqa34b", 1), ("swapstress", 1)])
+def test_sgmv_parity(H, name, shrink):
+    """shrink = 1: the mma.sync shrink also where long segments above rank 16 would take the tcgen05 one."""
+    from paper_2505_03756_b200 import binding as fl
     wl = synth.make_workload(name, **REDUCED[name])
     s = _session(H, wl)
     try:
+        fl.fl_pool_set_option(s.pool, fl.FL_OPT_SGMV_SHRINK, shrink)
         seg, ids = wl.segments()
         groups = [["q", "k", "v"], ["o"]] + ([["up"], ["down"]] if wl.shape.inter else [])
         for grp in groups:

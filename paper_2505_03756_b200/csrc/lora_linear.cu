@@ -44,16 +44,16 @@ template <int BN>
 struct Cfg {
   static constexpr uint32_t B_BYTES = (BN / 64) * B_GROUP;
   static constexpr uint32_t STAGE = A_BYTES + B_BYTES;
-  static constexpr int NS = BN == 256 ? 4 : 6;
+  static constexpr int NS = BN == 256 ? 4 : BN == 128 ? 5 : 6;
   // a LoRA stage: v tile [128 x 32 ranks] in 128-byte rows (half of each row used) + B rows [32 x BN]
   static constexpr uint32_t EB_GROUP = ER * 128;
   static constexpr uint32_t EXT = A_BYTES + (BN / 64) * EB_GROUP;
-  static constexpr int NE = BN == 256 ? 1 : 4;
+  static constexpr int NE = BN == 256 ? 1 : BN == 128 ? 2 : 4;
   static constexpr uint32_t OFF_EXT = NS * STAGE;
   static constexpr uint32_t OFF_BAR = OFF_EXT + NE * EXT;
   static constexpr uint32_t SMEM = OFF_BAR + 256 + 1024;      // barriers and bookkeeping; slack for 1024-byte alignment
   static constexpr uint32_t TMEM_COLS = 2 * BN;               // two accumulators
-  static_assert(TMEM_COLS == 512 || TMEM_COLS == 128, "TMEM allocations are powers of two");
+  static_assert(TMEM_COLS == 512 || TMEM_COLS == 256 || TMEM_COLS == 128, "TMEM allocations are powers of two");
   static_assert(SMEM <= 227 * 1024, "shared memory");
   static_assert(EXT % 1024 == 0 && STAGE % 1024 == 0, "operand tiles start on 1024-byte boundaries");
 };
@@ -443,6 +443,17 @@ int launch_linear(fl_pool* p, const LinArgs& a, const LinMaps& maps, cudaStream_
   return FL_OK;
 }
 
+int launch_width(fl_pool* p, const LinArgs& a, const LinMaps& maps, cudaStream_t st, int bn, int rmax) {
+  if (bn == 256)
+    return rmax == 16 ? launch_linear<256, 16>(p, a, maps, st)
+         : rmax == 32 ? launch_linear<256, 32>(p, a, maps, st) : launch_linear<256, 64>(p, a, maps, st);
+  if (bn == 128)
+    return rmax == 16 ? launch_linear<128, 16>(p, a, maps, st)
+         : rmax == 32 ? launch_linear<128, 32>(p, a, maps, st) : launch_linear<128, 64>(p, a, maps, st);
+  return rmax == 16 ? launch_linear<64, 16>(p, a, maps, st)
+       : rmax == 32 ? launch_linear<64, 32>(p, a, maps, st) : launch_linear<64, 64>(p, a, maps, st);
+}
+
 }  // namespace
 
 extern "C" {
@@ -536,12 +547,23 @@ int linear_common(fl_pool* p, fl_bf16* const* ys_in, const fl_bf16* x, const fl_
     a.n_kv = kv->n_kv;
     a.bt = (int)(p->block_bytes / per_tok);
   }
-  // few token tiles: narrower column tiles, so that every SM streams a slice of W
+  // few token tiles: narrower column tiles, so that every SM streams a slice of W.  Among 256, 128 and 64 columns the
+  // width with the least bytes through the busiest SM wins: rounds of tiles over the SMs times what a tile pulls per
+  // k-stage (its W slice and its x rows).
   int bn = 256;
   {
-    long tiles256 = 0;
-    for (int j = 0; j < n_mats; ++j) tiles256 += (long)lw.m_tiles * ((a.d_out[j] + 255) / 256);
-    if (tiles256 < p->sm_count || hybrid) bn = 64;
+    auto tiles = [&](int w) {
+      long t = 0;
+      for (int j = 0; j < n_mats; ++j) t += (long)lw.m_tiles * ((a.d_out[j] + w - 1) / w);
+      return t;
+    };
+    if (tiles(256) < p->sm_count || hybrid) {
+      long best = -1;
+      for (int w = 256; w >= 64; w /= 2) {
+        const long cost = ((tiles(w) + p->sm_count - 1) / p->sm_count) * (w + BM);
+        if (best < 0 || cost < best) { best = cost; bn = w; }
+      }
+    }
   }
   a.tile_base[0] = 0;
   for (int j = 0; j < n_mats; ++j) {
@@ -589,8 +611,7 @@ int linear_common(fl_pool* p, fl_bf16* const* ys_in, const fl_bf16* x, const fl_
       // y = x W from the GEMM alone, then the segmented projection adds the LoRA term to it
       a.ksplit = 1;
       a.rmax = info.rmax;
-      rc = info.rmax == 16 ? launch_linear<64, 16>(p, a, maps, st) : info.rmax == 32 ? launch_linear<64, 32>(p, a, maps, st)
-                                                                                   : launch_linear<64, 64>(p, a, maps, st);
+      rc = launch_width(p, a, maps, st, bn, info.rmax);
       if (rc != FL_OK) break;
       if (kv && n_mats == 3 && kv->k_slot == 1 && kv->v_slot == 2)
         rc = fl_lora_sgmv_qkv_append(p, ys[0], ys[1], ys[2], x, mat_indices[0], mat_indices[1], mat_indices[2], seg_indptr,
@@ -611,12 +632,7 @@ int linear_common(fl_pool* p, fl_bf16* const* ys_in, const fl_bf16* x, const fl_
     }
     a.ksplit = info.ksplit;
     a.rmax = info.rmax;
-    if (bn == 256)
-      rc = info.rmax == 16 ? launch_linear<256, 16>(p, a, maps, st)
-         : info.rmax == 32 ? launch_linear<256, 32>(p, a, maps, st) : launch_linear<256, 64>(p, a, maps, st);
-    else
-      rc = info.rmax == 16 ? launch_linear<64, 16>(p, a, maps, st)
-         : info.rmax == 32 ? launch_linear<64, 32>(p, a, maps, st) : launch_linear<64, 64>(p, a, maps, st);
+    rc = launch_width(p, a, maps, st, bn, info.rmax);
   } while (0);
   if (prev != p->device && prev >= 0) cudaSetDevice(prev);
   return rc;

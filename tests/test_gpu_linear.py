@@ -214,3 +214,28 @@ def test_fused_layer_replayed_from_cuda_graph_is_bit_identical(H):
         assert s.status()["device_flags"] == 0
     finally:
         s.close()
+
+
+@pytest.mark.parametrize("name,kw", [("decode13b", dict(n_req=200, len_range=(30, 90), n_adapters=20)),
+                                     ("prefill7b", dict(n_req=2, len_range=(400, 600), n_adapters=2))])
+def test_lora_linear_mid_sized_batches(H, name, kw):
+    """Batches between the decode and the prefill regime: a few token tiles, so the call picks 128-column tiles (with
+    LoRA stages for the long segments, without them for the batch of one-token segments)."""
+    wl = synth.make_workload(name, **kw)
+    s = _session(H, wl)
+    try:
+        seg, ids = wl.segments()
+        d_out = dict((n, o) for n, _, o in wl.shape.mats)
+        for grp in _groups(wl):
+            x = wl.x(grp[0])
+            tx = H.f32_to_dev(x, s.dev)
+            tw = [H.f32_to_dev(wl.weight(m), s.dev) for m in grp]
+            ty = [torch.full((wl.n_tokens, d_out[m]), 3.0, dtype=torch.bfloat16, device=s.dev) for m in grp]
+            s.lora_linear(ty, tx, tw, grp)
+            torch.cuda.synchronize()
+            for m, t in zip(grp, ty):
+                want = lora_linear(x, wl.weight(m), seg, ids, oracle_adapters(wl, m), wl.scale)
+                assert_close(H.dev_to_f32(t), want, f"{name}/mid-sized linear {m}")
+        assert s.status()["device_flags"] == 0
+    finally:
+        s.close()

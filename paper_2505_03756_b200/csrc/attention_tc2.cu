@@ -9,7 +9,8 @@
 //   warps 0-3   softmax of tile A (thread = query row = TMEM lane)      warp 8   TMA producer, unit fetch
 //   warps 4-7   softmax of tile B                                        warp 9   MMA issuer, TMEM owner
 //   (warps 10, 11 only complete the third warpgroup, whose registers go to the softmax warpgroups)
-//   K_j / V_j (128 keys = 8 pool pages each) -> ring of 32 KiB slots, 128-byte swizzle
+//   K_j / V_j (128 keys = 8 pool pages each, one 4 KiB TMA box per page) -> ring of 32 KiB slots, 128-byte swizzle;
+//   a page lands as [8-key group][64-value half][8 keys][64 values], so a tile's 8-key groups are 2 KiB apart
 //   S_X = Q_X K_j^T     tcgen05.mma 128x128x16 (x8) into TMEM columns of tile X
 //   P_X = exp2(S_X - m) -> bf16 pairs written back over the first half of S_X in TMEM
 //   O_X += P_X V_j      tcgen05.mma with the A operand read from TMEM, V MN-major as stored
@@ -38,6 +39,8 @@ constexpr int KT2 = 128;                               // keys per tile
 constexpr int NSLOT = 5;                               // ring slots; fills go K_0, V_0, K_1, V_1, ... across units
 constexpr uint32_t HALF_BYTES = 128 * 128;             // [128 rows][64 bf16], swizzled
 constexpr uint32_t TILE_BYTES = 2 * HALF_BYTES;        // a Q, K or V tile
+constexpr uint32_t PAGE_BYTES = BT * 128 * 2;          // K or V of one head of one block: [2 groups][2 halves][8 tokens][64 bf16]
+constexpr uint32_t GROUP_BYTES = PAGE_BYTES / 2;       // stride between 8-key groups of a K/V tile
 constexpr uint32_t OFF_Q2 = 0;                         // Q_A, Q_B
 constexpr uint32_t OFF_RING = 2 * TILE_BYTES;
 constexpr uint32_t OFF_BAR2 = OFF_RING + NSLOT * TILE_BYTES;
@@ -156,8 +159,8 @@ attn_prefill_tc2_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap kv
     asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
     if (warp == 8) {
       // ------------------------------------------------ unit fetch + TMA producer
-      // The whole warp runs the loop; lane 0 fetches units and does the waiting, lanes 0-15 each own one half of one of a
-      // tile's eight pages (their block-id loads and their TMA issues run side by side).
+      // The whole warp runs the loop; lane 0 fetches units and does the waiting, lanes 0-7 each own one of a tile's eight
+      // pages (their block-id loads and their TMA issues run side by side).
       int fill = 0;                    // ring fills so far, over all units
       int n_valid = 0;                 // units whose Q tiles were loaded so far
       bool ok = true;
@@ -197,10 +200,10 @@ attn_prefill_tc2_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap kv
         for (int j = 0; ok && j < n_kt_max; ++j) {
           // this lane's page of the tile (pages behind the last needed key are masked anyway: re-read the last
           // valid page); K_j and V_j come from the same blocks
-          // lane = 2 * page + half: sixteen lanes issue one box each
+          // lane = page: eight lanes issue one 4 KiB box each
           uint32_t blk = 0;
-          if (lane < 2 * (KT2 / BT)) {
-            blk = a.tbl[tbl0 + min(j * (KT2 / BT) + (lane >> 1), n_pages - 1)];
+          if (lane < KT2 / BT) {
+            blk = a.tbl[tbl0 + min(j * (KT2 / BT) + lane, n_pages - 1)];
             if (blk >= a.pv.n_blocks) {
               atomicOr(a.pv.flags, (uint32_t)FLAG_BAD_BLOCK);
               blk = 0;
@@ -215,11 +218,9 @@ attn_prefill_tc2_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap kv
             }
             ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;     // the transaction count is armed before any copy is issued
             if (!ok) break;
-            if (lane < 2 * (KT2 / BT)) {
-              const int page = lane >> 1, half = lane & 1;
-              const uint32_t dst = sbase + OFF_RING + s * TILE_BYTES + half * HALF_BYTES + page * (BT * 128);
-              tma_load_4d(dst, &kv_map, bar(C_FULL + s), 64 * half, 0, side * a.n_kv + h, (int)blk);
-            }
+            if (lane < KT2 / BT)
+              tma_load_5d(sbase + OFF_RING + s * TILE_BYTES + lane * PAGE_BYTES, &kv_map, bar(C_FULL + s), 0, 0, 0,
+                          2 * (side * a.n_kv + h), (int)blk);
           }
         }
       }
@@ -236,8 +237,9 @@ attn_prefill_tc2_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap kv
         const uint32_t qb = sbase + OFF_Q2 + x * TILE_BYTES, kb = slot_addr(kslot);
 #pragma unroll
         for (int ks = 0; ks < D / 16; ++ks) {
-          const uint32_t off = (ks >> 2) * HALF_BYTES + (ks & 3) * 32;
-          umma_bf16(tmem + x * 128, smem_desc(qb + off, 16, 1024), smem_desc(kb + off, 16, 1024), IDESC, ks > 0);
+          // Q: [half][128 rows][128 B]; K: eight pages, each [group][half][8 keys][128 B]
+          umma_bf16(tmem + x * 128, smem_desc(qb + (ks >> 2) * HALF_BYTES + (ks & 3) * 32, 16, 1024),
+                    smem_desc(kb + (ks >> 2) * 1024 + (ks & 3) * 32, 16, GROUP_BYTES), IDESC, ks > 0);
         }
         umma_commit(bar(C_SFULL + x));
       };
@@ -245,8 +247,8 @@ attn_prefill_tc2_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap kv
         const uint32_t vb = slot_addr(vslot);
 #pragma unroll
         for (int ks = 0; ks < KT2 / 16; ++ks)
-          umma_bf16_ts(tmem + 256 + x * 128, tmem + x * 128 + ks * 8, smem_desc(vb + ks * (16 * 128), HALF_BYTES, 1024),
-                       IDESC_PV, (!first || ks > 0));
+          umma_bf16_ts(tmem + 256 + x * 128, tmem + x * 128 + ks * 8, smem_desc(vb + ks * PAGE_BYTES, 1024, GROUP_BYTES),
+                       IDESC_PV, (!first || ks > 0));   // 16 keys = one page; halves 1 KiB apart, groups 2 KiB apart
         if (last) umma_commit(bar(C_ODONE + x));
       };
       bool ok = true;

@@ -55,11 +55,14 @@ int kv_pages(fl_pool* p, int n_kv, const CUtensorMap** out) {
       tc->n_kv = -1;
       p->tmap_cache = tc;
     }
-    const uint64_t dims[4] = {(uint64_t)FL_HEAD_DIM, 16, (uint64_t)(2 * n_kv), (uint64_t)p->n_blocks};
-    const uint64_t strides[3] = {(uint64_t)FL_HEAD_DIM * 2, (uint64_t)16 * FL_HEAD_DIM * 2, (uint64_t)p->block_bytes};
-    const uint32_t box[4] = {64, 16, 1, 1};
+    // One box = K (or V) of one head of one block, 16 tokens x 128 values = 4 KiB, written to shared memory as
+    // [8-token group][64-value half][token][64 values]: coordinates {value, token in group, half, 2 KiB chunk of the
+    // block, block}; a chunk is one 8-token group of one (K|V, head) plane.
+    const uint64_t dims[5] = {64, 8, 2, (uint64_t)(4 * n_kv), (uint64_t)p->n_blocks};
+    const uint64_t strides[4] = {(uint64_t)FL_HEAD_DIM * 2, 128, (uint64_t)8 * FL_HEAD_DIM * 2, (uint64_t)p->block_bytes};
+    const uint32_t box[5] = {64, 8, 2, 2, 1};
     tc->n_kv = -1;
-    if (encode_bf16(&tc->kv, p->slab, 4, dims, strides, box) != FL_OK) return FL_ECUDA;
+    if (encode_bf16(&tc->kv, p->slab, 5, dims, strides, box) != FL_OK) return FL_ECUDA;
     tc->n_kv = n_kv;
   }
   *out = &tc->kv;

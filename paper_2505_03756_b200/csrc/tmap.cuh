@@ -12,8 +12,8 @@ namespace tmap {
 int encode_bf16(CUtensorMap* out, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
                 const uint32_t* box);
 
-// The slab as [block][K|V x kv head][token][128] with a box of one 64-element half of a 16-token page
-// (cached in the pool, keyed by the KV head count).
+// The slab as [block][K|V x kv head][token][128] with a box of one 16-token page of one plane (4 KiB), laid out in
+// shared memory as [8-token group][64-value half][8 tokens][64 values] (cached in the pool, keyed by the KV head count).
 int kv_pages(fl_pool* p, int n_kv, const CUtensorMap** out);
 
 }  // namespace tmap

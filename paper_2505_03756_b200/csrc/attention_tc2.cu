@@ -144,14 +144,6 @@ attn_prefill_tc2_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap kv
   const int n_units = a.hdr->n_prefill * heads_per_item;   // a CTA beyond the last unit finds no work and tears down
 
   // Readers take the k-th unit of this CTA from slot k & 1 (index -1 = no more work) and release the slot.
-  auto read_unit = [&](int k, bool arrive) -> Unit {
-    Unit t;
-    t.index = -1;
-    if (!mbar_wait(bar(C_UFULL + (k & 1)), (k >> 1) & 1, abort_flag)) return t;
-    t = unit_slot[k & 1];
-    if (arrive) mbar_arrive(bar(C_UEMPTY + (k & 1)));
-    return t;
-  };
 
   // the softmax warpgroups keep 128 scores per thread in registers: they take the registers the third
   // warpgroup does not need
@@ -224,54 +216,63 @@ attn_prefill_tc2_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap kv
           }
         }
       }
-    } else if (warp == 9 && lane == 0) {
+    } else if (warp == 9) {
       // ------------------------------------------------ MMA issuer
+      // The whole warp runs the loop converged and an elected lane issues each MMA and commit, so that descriptors and
+      // addresses depend on nothing lane-specific; a descriptor is a fixed high word and a low word that steps by adds.
       constexpr uint32_t IDESC = instr_desc(128, false);        // S: both operands K-major
       constexpr uint32_t IDESC_PV = instr_desc(D, true);        // O: V is MN-major
+      constexpr uint32_t HI_Q = desc_hi(1024), HI_KV = desc_hi(GROUP_BYTES);
+      const uint32_t q_lo[2] = {desc_lo(sbase + OFF_Q2, 16), desc_lo(sbase + OFF_Q2 + TILE_BYTES, 16)};
+      const uint32_t ring_k_lo = desc_lo(sbase + OFF_RING, 16), ring_v_lo = desc_lo(sbase + OFF_RING, 1024);
       int cons = 0;                    // ring slots consumed so far, over all units
       int steps[2] = {0, 0};           // P tiles awaited so far per tile (phase of C_PFULL)
       int n_done = 0;                  // valid units so far (phase of C_QFULL)
-      auto slot_addr = [&](int idx) { return sbase + OFF_RING + (idx % NSLOT) * TILE_BYTES; };
-      auto wait_full = [&](int idx) { return mbar_wait(bar(C_FULL + idx % NSLOT), (idx / NSLOT) & 1, abort_flag); };
+      auto wait_all = [&](uint32_t b, uint32_t parity) { return __all_sync(0xffffffffu, mbar_wait(b, parity, abort_flag)) != 0; };
+      auto slot_off = [&](int idx) { return (uint32_t)(idx % NSLOT) * (TILE_BYTES >> 4); };
+      auto wait_full = [&](int idx) { return wait_all(bar(C_FULL + idx % NSLOT), (idx / NSLOT) & 1); };
       auto issue_s = [&](int x, int kslot) {
-        const uint32_t qb = sbase + OFF_Q2 + x * TILE_BYTES, kb = slot_addr(kslot);
+        const uint32_t k_lo = ring_k_lo + slot_off(kslot);
 #pragma unroll
         for (int ks = 0; ks < D / 16; ++ks) {
           // Q: [half][128 rows][128 B]; K: eight pages, each [group][half][8 keys][128 B]
-          umma_bf16(tmem + x * 128, smem_desc(qb + (ks >> 2) * HALF_BYTES + (ks & 3) * 32, 16, 1024),
-                    smem_desc(kb + (ks >> 2) * 1024 + (ks & 3) * 32, 16, GROUP_BYTES), IDESC, ks > 0);
+          umma_ss_elect(tmem + x * 128, q_lo[x] + (((ks >> 2) * HALF_BYTES + (ks & 3) * 32) >> 4), HI_Q,
+                        k_lo + (((ks >> 2) * 1024 + (ks & 3) * 32) >> 4), HI_KV, IDESC, ks > 0);
         }
-        umma_commit(bar(C_SFULL + x));
+        umma_commit_elect(bar(C_SFULL + x));
       };
       auto issue_pv = [&](int x, int vslot, bool first, bool last) {
-        const uint32_t vb = slot_addr(vslot);
+        const uint32_t v_lo = ring_v_lo + slot_off(vslot);
 #pragma unroll
-        for (int ks = 0; ks < KT2 / 16; ++ks)
-          umma_bf16_ts(tmem + 256 + x * 128, tmem + x * 128 + ks * 8, smem_desc(vb + ks * PAGE_BYTES, 1024, GROUP_BYTES),
-                       IDESC_PV, (!first || ks > 0));   // 16 keys = one page; halves 1 KiB apart, groups 2 KiB apart
-        if (last) umma_commit(bar(C_ODONE + x));
+        for (int ks = 0; ks < KT2 / 16; ++ks)   // 16 keys = one page; halves 1 KiB apart, groups 2 KiB apart
+          umma_ts_elect(tmem + 256 + x * 128, tmem + x * 128 + ks * 8, v_lo + ks * (PAGE_BYTES >> 4), HI_KV, IDESC_PV,
+                        (!first || ks > 0));
+        if (last) umma_commit_elect(bar(C_ODONE + x));
       };
       bool ok = true;
       for (int k = 0; ok; ++k) {
-        const Unit t = read_unit(k, true);
+        if (!wait_all(bar(C_UFULL + (k & 1)), (k >> 1) & 1)) break;
+        const Unit t = unit_slot[k & 1];
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar(C_UEMPTY + (k & 1)));
         if (t.index < 0) break;
         if (!t.valid) continue;
         const int n_kt = t.n_kt_max, nA = t.n_kt[0], nB = t.n_kt[1];
         const int base = cons;         // ring index of K_0 of this unit; K_j = base + 2j, V_j = base + 2j + 1
-        ok = mbar_wait(bar(C_QFULL), n_done & 1, abort_flag) && wait_full(base);
+        ok = wait_all(bar(C_QFULL), n_done & 1) && wait_full(base);
         if (!ok) break;
         ++n_done;
         tc_fence_after();
         if (nA > 0) issue_s(0, base);
         if (nB > 0) issue_s(1, base);
-        umma_commit(bar(C_EMPTY + base % NSLOT));
-        if (n_kt == 1) umma_commit(bar(C_QEMPTY));
+        umma_commit_elect(bar(C_EMPTY + base % NSLOT));
+        if (n_kt == 1) umma_commit_elect(bar(C_QEMPTY));
         for (int j = 0; ok && j < n_kt; ++j) {
           const bool more = j + 1 < n_kt;
           const int vs = base + 2 * j + 1, kn = base + 2 * j + 2;
           ok = wait_full(vs);
           if (ok && j < nA) {
-            ok = mbar_wait(bar(C_PFULL + 0), steps[0]++ & 1, abort_flag);
+            ok = wait_all(bar(C_PFULL + 0), steps[0]++ & 1);
             if (ok) { tc_fence_after(); issue_pv(0, vs, j == 0, j == nA - 1); }
           }
           if (ok && more) ok = wait_full(kn);
@@ -279,15 +280,15 @@ attn_prefill_tc2_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap kv
           tc_fence_after();
           if (j + 1 < nA) issue_s(0, kn);
           if (j < nB) {
-            ok = mbar_wait(bar(C_PFULL + 1), steps[1]++ & 1, abort_flag);
+            ok = wait_all(bar(C_PFULL + 1), steps[1]++ & 1);
             if (!ok) break;
             tc_fence_after();
             issue_pv(1, vs, j == 0, j == nB - 1);
           }
-          umma_commit(bar(C_EMPTY + vs % NSLOT));
+          umma_commit_elect(bar(C_EMPTY + vs % NSLOT));
           if (j + 1 < nB) issue_s(1, kn);
-          if (more) umma_commit(bar(C_EMPTY + kn % NSLOT));
-          if (j + 2 == n_kt) umma_commit(bar(C_QEMPTY));     // the unit's last S MMAs are in the pipe: Q is free after them
+          if (more) umma_commit_elect(bar(C_EMPTY + kn % NSLOT));
+          if (j + 2 == n_kt) umma_commit_elect(bar(C_QEMPTY));     // the unit's last S MMAs are in the pipe: Q is free after them
         }
         cons = base + 2 * n_kt;
       }

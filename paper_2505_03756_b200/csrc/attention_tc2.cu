@@ -52,6 +52,12 @@ enum { C_QFULL = 0, C_QEMPTY = 1, C_FULL = 2, C_EMPTY = C_FULL + NSLOT, C_SFULL 
        C_ODONE = C_PFULL + 2, C_UFULL = C_ODONE + 2, C_UEMPTY = C_UFULL + 2, C_COUNT = C_UEMPTY + 2 };
 constexpr int UNIT_READERS = 9;                        // MMA issuer + 8 softmax warps
 
+// 32 bytes to a 32-byte aligned global address in one instruction.
+__device__ __forceinline__ void st_global_v8(void* dst, const uint32_t* r) {
+  asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(dst), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]),
+               "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]) : "memory");
+}
+
 struct Unit {           // what a CTA works on at one time
   int tok0[2];          // first token row (in the packed q / out tensors) of each tile
   int hq[2];            // query head of each tile
@@ -98,7 +104,7 @@ __device__ __forceinline__ Unit decode_unit(const AttnArgs& a, int u, int heads_
 
 __global__ void __launch_bounds__(T2_THREADS, 1)
 attn_prefill_tc2_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap kv_map, const __grid_constant__ CUtensorMap q_map,
-                        int heads_per_item) {
+                        int heads_per_item, int wide_out) {
   extern __shared__ __align__(1024) unsigned char smem[];
   const uint32_t sbase = smem_u32(smem);
   if (sbase & 1023u) {   // the swizzled operand tiles need 1024-byte alignment
@@ -382,7 +388,7 @@ attn_prefill_tc2_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap kv
         __syncwarp();
         if (lane == 0) mbar_arrive(bar(C_PFULL + x));
       }
-      // ---- epilogue: O / l -> bf16, each thread stores its own row (16 x 16 bytes, contiguous)
+      // ---- epilogue: O / l -> bf16, each thread stores its own row (8 x 32 bytes, contiguous)
       if (ok) ok = mbar_wait(bar(C_ODONE + x), epis++ & 1, abort_flag);
       if (!ok) break;
       tc_fence_after();
@@ -394,14 +400,15 @@ attn_prefill_tc2_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap kv
         tmem_ld32(o_addr + cb, o);
         tmem_wait_ld();
         if (row < rows) {
+          uint32_t pk[16];
 #pragma unroll
-          for (int c = 0; c < 4; ++c) {
-            uint4 v;
-            v.x = pack_bf16(__uint_as_float(o[8 * c + 0]) * inv, __uint_as_float(o[8 * c + 1]) * inv);
-            v.y = pack_bf16(__uint_as_float(o[8 * c + 2]) * inv, __uint_as_float(o[8 * c + 3]) * inv);
-            v.z = pack_bf16(__uint_as_float(o[8 * c + 4]) * inv, __uint_as_float(o[8 * c + 5]) * inv);
-            v.w = pack_bf16(__uint_as_float(o[8 * c + 6]) * inv, __uint_as_float(o[8 * c + 7]) * inv);
-            orow[(cb >> 3) + c] = v;
+          for (int c = 0; c < 16; ++c) pk[c] = pack_bf16(__uint_as_float(o[2 * c]) * inv, __uint_as_float(o[2 * c + 1]) * inv);
+          if (wide_out) {                              // 32 bytes per lane: half as many store instructions per row
+            st_global_v8(orow + (cb >> 3), pk);
+            st_global_v8(orow + (cb >> 3) + 2, pk + 8);
+          } else {
+#pragma unroll
+            for (int c = 0; c < 4; ++c) orow[(cb >> 3) + c] = make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
           }
         }
       }
@@ -455,7 +462,8 @@ int launch_prefill_tc2(fl_pool* p, const AttnArgs& a, int n_tokens, int max_item
   const long long units = (long long)max_items * heads_per_item;
   const unsigned grid = (unsigned)std::min<long long>(units, p->sm_count);
   if (grid == 0) return FL_OK;
-  FL_CUDA(p, launch_pdl(attn_prefill_tc2_kernel, dim3(grid), dim3(T2_THREADS), T2_SMEM, st, a, *kv, qmap, heads_per_item));
+  FL_CUDA(p, launch_pdl(attn_prefill_tc2_kernel, dim3(grid), dim3(T2_THREADS), T2_SMEM, st, a, *kv, qmap, heads_per_item,
+                     (reinterpret_cast<uintptr_t>(a.out) & 31) == 0 ? 1 : 0));   // 32-byte stores where the output allows them
   FL_CUDA(p, cudaGetLastError());
   return FL_OK;
 }

@@ -93,8 +93,15 @@ __global__ void __launch_bounds__(256) attn_plan_kernel(const AttnArgs a, int ch
     if (n <= 0 || n * group <= DEC_ROWS) continue;
     const int tiles = (n + qt - 1) / qt;
     const int first = atomicAdd(&cursor[key_of(i)], tiles);
-    for (int t = 0; t < tiles; ++t)
-      if (first + t < a.max_prefill) a.prefill_list[first + t] = make_int2(i, (tiles - 1 - t) * qt);
+    // An item of 256 tokens is two 128-row tiles that share one K/V stream and costs as many key tiles as its later
+    // tile needs.  With an odd number of 128-row tiles the request's FIRST tile (shortest context) goes alone and the
+    // pairs start at token 128, instead of the last tile (longest context) going alone: one key tile less per pair.
+    const bool lone_first = qt == 256 && (((n + 127) / 128) & 1);
+    for (int t = 0; t < tiles; ++t) {
+      const int u = tiles - 1 - t;      // item number in token order
+      const int q0 = lone_first ? (u == 0 ? 0 : 128 + (u - 1) * 256) : u * qt;
+      if (first + t < a.max_prefill) a.prefill_list[first + t] = make_int2(i, q0);
+    }
   }
   if (threadIdx.x == 0) {
     if (base_p > a.max_prefill || base_d > a.max_decode) atomicOr(a.pv.flags, (uint32_t)FLAG_BAD_POS);

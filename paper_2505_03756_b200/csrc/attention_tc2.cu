@@ -88,7 +88,9 @@ __device__ __forceinline__ Unit decode_unit(const AttnArgs& a, int u, int heads_
     t.hq[0] = t.hq[1] = hslot;
     t.h = hslot / group;
     t.tok0[0] = a.req_indptr[i] + q0; t.tok0[1] = t.tok0[0] + 128;
-    t.rows[0] = min(128, n_new - q0); t.rows[1] = max(0, min(128, n_new - q0 - 128));
+    // a request with an odd number of 128-row tiles has its first tile alone (the plan starts its pairs at token 128)
+    const bool lone = q0 == 0 && (((n_new + 127) / 128) & 1);
+    t.rows[0] = min(128, n_new - q0); t.rows[1] = lone ? 0 : max(0, min(128, n_new - q0 - 128));
     t.lim0[0] = prefix + q0; t.lim0[1] = prefix + q0 + 128;
   }
 #pragma unroll

@@ -281,8 +281,9 @@ int fl_kv_append(fl_pool* pool, const fl_bf16* k_new, const fl_bf16* v_new, cons
  * reused as stored, the new tokens (already appended) are causal.  Prefill, decode (new_len 1) and
  * mixed batches go through the same call.  q, out: device [n_tokens, n_q_heads, 128] bf16 packed by
  * request (req_indptr); new_lens[i] = req_indptr[i+1] - req_indptr[i].  n_tbl = total number of
- * table entries.  Needs block tokens bt = 16.  workspace: device scratch of at least
- * fl_paged_attention_workspace(...) bytes; same sharing rule as above. */
+ * table entries.  Needs block tokens bt = 16.  out on a 32-byte boundary lets the prefill kernel store 32 bytes per
+ * instruction (16-byte alignment, the general rule, is enough; the result is the same).  workspace: device scratch of at
+ * least fl_paged_attention_workspace(...) bytes; same sharing rule as above. */
 size_t fl_paged_attention_workspace(int n_req, int n_tokens, int n_tbl, int n_q_heads, int n_kv_heads);
 int fl_paged_attention(fl_pool* pool, fl_bf16* out, const fl_bf16* q, const int32_t* req_indptr,
                        const int32_t* kv_tbl_indptr, const uint32_t* kv_tbl, const int32_t* prefix_lens,

@@ -494,3 +494,39 @@ def test_attention_unusual_head_groupings(H, heads):
     wl.pool_blocks = 160
     for kernel in (0, 1):
         _attention_case(H, wl, prefill_kernel=kernel)
+
+
+def test_attention_odd_tile_counts_without_grouped_heads(H):
+    # one head per KV head: a unit pairs two consecutive 128-row tiles of a request; with 1, 3, 5 and 7 tiles the first
+    # tile goes alone and the pairs start at token 128, with 2 and 4 tiles they start at token 0; ragged last tiles
+    sh = synth.LayerShape(512, 4, 4)
+    wl = synth.make_workload("tiny", n_req=6, len_range=(0, 0), n_adapters=1, shape=sh)
+    wl.prefix_lens[:] = [0, 130, 16, 300, 0, 77]
+    wl.new_lens[:] = [100, 300, 256, 640, 512, 800]
+    wl.pool_blocks = 320
+    _attention_case(H, wl)
+
+
+def test_attention_output_on_a_16_byte_boundary(H):
+    """The output pointer must be 16-byte aligned; on a 32-byte boundary the tensor-core kernel stores 32 bytes per
+    instruction, otherwise 16: the two paths give the same bits."""
+    wl = synth.make_workload("prefill7b", n_req=2, len_range=(150, 400))
+    want = _attention_case(H, wl)
+    s = H.Session(wl, adapters=[])
+    try:
+        s.build_batch()
+        s.fill_prefix_kv()
+        k_new, v_new = wl.kv_new()
+        q = wl.q()
+        s.kv_append(H.f32_to_dev(k_new, s.dev), H.f32_to_dev(v_new, s.dev))
+        n = int(np.prod(q.shape))
+        buf = torch.zeros(n + 8, dtype=torch.bfloat16, device=s.dev)
+        out = buf[8:].view(wl.n_tokens, -1)
+        assert out.data_ptr() % 32 == 16
+        s.attention(out, H.f32_to_dev(q, s.dev))
+        torch.cuda.synchronize()
+        assert np.array_equal(H.dev_to_f32(out).reshape(want.shape), want)
+        assert float(buf[:8].float().abs().sum()) == 0.0
+        assert s.status()["device_flags"] == 0
+    finally:
+        s.close()

@@ -513,10 +513,53 @@ def bench_workload(args, name, world, rank, local, oracle_budget_s):
             h_out.copy_(d_z["down" if s.inter else "o"].view(torch.int16), non_blocking=True)
         for k in range(2):
             e2e_step(k)
-        ms_e2e = timed(e2e_step, max(3, min(args.steps, 20)))
+        ms_e2e_serial = timed(e2e_step, max(3, min(args.steps, 20)))
+
+        # the same with consecutive steps pipelined, as a server would run them: while step k computes, the x of step k + 1
+        # is on its way up and the output of step k - 1 on its way down (two staging buffers each way, three streams)
+        up, down = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)
+        out_t = d_z["down" if s.inter else "o"]
+        st_in = [torch.empty_like(d_x) for _ in range(2)]
+        st_out = [torch.empty_like(out_t) for _ in range(2)]
+        pev = {n: [torch.cuda.Event() for _ in range(2)] for n in ("up", "in_free", "comp", "down")}
+
+        def e2e_pipelined(k):
+            b = k & 1
+            if k >= 2:
+                up.wait_event(pev["in_free"][b])
+            with torch.cuda.stream(up):
+                st_in[b].view(torch.int16).copy_(h_x, non_blocking=True)
+                pev["up"][b].record(up)
+            main.wait_event(pev["up"][b])
+            d_x.copy_(st_in[b], non_blocking=True)
+            pev["in_free"][b].record(main)
+            step(0, use_graph=True, fused=True)
+            if k >= 2:
+                main.wait_event(pev["down"][b])
+            st_out[b].copy_(out_t, non_blocking=True)
+            pev["comp"][b].record(main)
+            down.wait_event(pev["comp"][b])
+            with torch.cuda.stream(down):
+                h_out.copy_(st_out[b].view(torch.int16), non_blocking=True)
+                pev["down"][b].record(down)
+
+        def timed_pipeline(n):
+            barrier()
+            t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            t0.record(main)
+            for k in range(n):
+                e2e_pipelined(k)
+            for b in range(min(n, 2)):          # the last read-backs end the timed region
+                main.wait_event(pev["down"][b])
+            t1.record(main)
+            barrier()
+            return t0.elapsed_time(t1) / n
+        timed_pipeline(3)
+        ms_e2e = timed_pipeline(max(6, min(args.steps, 20)))
+        del st_in, st_out
     st = sess.status()
     flags = st["device_flags"]
-    (ms_step, ms_fused, ms_e2e), tokens_all = reduce_over_ranks([ms_step, ms_fused, ms_e2e], T, world, dev)
+    (ms_step, ms_fused, ms_e2e, ms_e2e_serial), tokens_all = reduce_over_ranks([ms_step, ms_fused, ms_e2e, ms_e2e_serial], T, world, dev)
     rec = None
     if rank == 0:
         pk = peaks()
@@ -583,8 +626,10 @@ def bench_workload(args, name, world, rank, local, oracle_budget_s):
             "cpu_baseline": cb,
             "e2e": {"value": tokens_all / (ms_e2e * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": int(h_x.numel() * 2),
                     "d2h_bytes_per_step": int(h_out.numel() * 2), "ms_per_step": ms_e2e,
-                    "step": "layer with base projections (fl_lora_linear), x uploaded from pinned host memory, "
-                            "the layer's output read back"},
+                    "ms_per_step_one_at_a_time": ms_e2e_serial,
+                    "step": "layer with base projections (fl_lora_linear), x uploaded from pinned host memory, the layer's "
+                            "output read back, every step; consecutive steps pipelined (upload of the next and read-back "
+                            "of the previous overlap the kernels); one_at_a_time = upload, kernels, read-back in sequence"},
             "gpu_launches": launches_per_step * args.steps, "launch_mode": launch_mode, "clocks": clocks, "device_flags": flags,
         }
     sess.close()

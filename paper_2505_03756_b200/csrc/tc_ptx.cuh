@@ -181,6 +181,60 @@ __device__ __forceinline__ void umma_commit_elect(uint32_t bar) {
       "elect.sync _|e, 0xffffffff;\n\t"
       "@e tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}" ::"r"(bar) : "memory");
 }
+// One 128 x 128 x 128 score tile as a single block: an elected lane of the converged warp issues the eight k-steps and the
+// commit.  Low descriptor words step by constants: Q is [half][128 rows][128 B] (k-steps 32 B apart, the halves 16 KiB),
+// K is eight pages of [8-key group][half][8 keys][128 B] (k-steps 32 B apart, the halves 1 KiB).
+__device__ __forceinline__ void umma_s_tile_elect(uint32_t d_tmem, uint32_t q_lo, uint32_t k_lo, uint32_t q_hi, uint32_t k_hi,
+                                                  uint32_t idesc, uint32_t commit_bar) {
+  asm volatile(
+      "{\n\t.reg .pred e, pt, pf;\n\t.reg .b64 da, db;\n\t.reg .b32 a, b;\n\t"
+      "elect.sync _|e, 0xffffffff;\n\t"
+      "setp.eq.u32 pt, 0, 0;\n\tsetp.ne.u32 pf, 0, 0;\n\t"
+      "add.u32 a, %1, 0;\n\tadd.u32 b, %2, 0;\n\tmov.b64 da, {a, %3};\n\tmov.b64 db, {b, %4};\n\t"
+      "@e tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, pf;\n\t"
+      "add.u32 a, %1, 2;\n\tadd.u32 b, %2, 2;\n\tmov.b64 da, {a, %3};\n\tmov.b64 db, {b, %4};\n\t"
+      "@e tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, pt;\n\t"
+      "add.u32 a, %1, 4;\n\tadd.u32 b, %2, 4;\n\tmov.b64 da, {a, %3};\n\tmov.b64 db, {b, %4};\n\t"
+      "@e tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, pt;\n\t"
+      "add.u32 a, %1, 6;\n\tadd.u32 b, %2, 6;\n\tmov.b64 da, {a, %3};\n\tmov.b64 db, {b, %4};\n\t"
+      "@e tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, pt;\n\t"
+      "add.u32 a, %1, 1024;\n\tadd.u32 b, %2, 64;\n\tmov.b64 da, {a, %3};\n\tmov.b64 db, {b, %4};\n\t"
+      "@e tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, pt;\n\t"
+      "add.u32 a, %1, 1026;\n\tadd.u32 b, %2, 66;\n\tmov.b64 da, {a, %3};\n\tmov.b64 db, {b, %4};\n\t"
+      "@e tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, pt;\n\t"
+      "add.u32 a, %1, 1028;\n\tadd.u32 b, %2, 68;\n\tmov.b64 da, {a, %3};\n\tmov.b64 db, {b, %4};\n\t"
+      "@e tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, pt;\n\t"
+      "add.u32 a, %1, 1030;\n\tadd.u32 b, %2, 70;\n\tmov.b64 da, {a, %3};\n\tmov.b64 db, {b, %4};\n\t"
+      "@e tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, pt;\n\t"
+      "@e tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%6];\n\t}"
+      ::"r"(d_tmem), "r"(q_lo), "r"(k_lo), "r"(q_hi), "r"(k_hi), "r"(idesc), "r"(commit_bar) : "memory");
+}
+// O (+)= P V for one 128-key tile: P as bf16 pairs in TMEM (8 columns per k-step), V as eight 4 KiB pages, one per k-step.
+__device__ __forceinline__ void umma_pv_tile_elect(uint32_t o_tmem, uint32_t p_tmem, uint32_t v_lo, uint32_t v_hi, uint32_t idesc,
+                                                   uint32_t accumulate_first) {
+  asm volatile(
+      "{\n\t.reg .pred e, pt, p0;\n\t.reg .b64 db;\n\t.reg .b32 a, b;\n\t"
+      "elect.sync _|e, 0xffffffff;\n\t"
+      "setp.eq.u32 pt, 0, 0;\n\tsetp.ne.u32 p0, %5, 0;\n\t"
+      "add.u32 a, %1, 0;\n\tadd.u32 b, %2, 0;\n\tmov.b64 db, {b, %3};\n\t"
+      "@e tcgen05.mma.cta_group::1.kind::f16 [%0], [a], db, %4, p0;\n\t"
+      "add.u32 a, %1, 8;\n\tadd.u32 b, %2, 256;\n\tmov.b64 db, {b, %3};\n\t"
+      "@e tcgen05.mma.cta_group::1.kind::f16 [%0], [a], db, %4, pt;\n\t"
+      "add.u32 a, %1, 16;\n\tadd.u32 b, %2, 512;\n\tmov.b64 db, {b, %3};\n\t"
+      "@e tcgen05.mma.cta_group::1.kind::f16 [%0], [a], db, %4, pt;\n\t"
+      "add.u32 a, %1, 24;\n\tadd.u32 b, %2, 768;\n\tmov.b64 db, {b, %3};\n\t"
+      "@e tcgen05.mma.cta_group::1.kind::f16 [%0], [a], db, %4, pt;\n\t"
+      "add.u32 a, %1, 32;\n\tadd.u32 b, %2, 1024;\n\tmov.b64 db, {b, %3};\n\t"
+      "@e tcgen05.mma.cta_group::1.kind::f16 [%0], [a], db, %4, pt;\n\t"
+      "add.u32 a, %1, 40;\n\tadd.u32 b, %2, 1280;\n\tmov.b64 db, {b, %3};\n\t"
+      "@e tcgen05.mma.cta_group::1.kind::f16 [%0], [a], db, %4, pt;\n\t"
+      "add.u32 a, %1, 48;\n\tadd.u32 b, %2, 1536;\n\tmov.b64 db, {b, %3};\n\t"
+      "@e tcgen05.mma.cta_group::1.kind::f16 [%0], [a], db, %4, pt;\n\t"
+      "add.u32 a, %1, 56;\n\tadd.u32 b, %2, 1792;\n\tmov.b64 db, {b, %3};\n\t"
+      "@e tcgen05.mma.cta_group::1.kind::f16 [%0], [a], db, %4, pt;\n\t"
+      "}"
+      ::"r"(o_tmem), "r"(p_tmem), "r"(v_lo), "r"(v_hi), "r"(idesc), "r"(accumulate_first) : "memory");
+}
 // Instruction descriptor: fp32 accumulate, bf16 x bf16, M = 128, N = n; b_mn = B operand is MN-major.
 __host__ __device__ constexpr uint32_t instr_desc(int n, bool b_mn) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn ? 1u : 0u) << 16) | ((uint32_t)(n >> 3) << 17) | ((128u >> 4) << 24);

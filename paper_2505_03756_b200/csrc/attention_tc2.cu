@@ -278,15 +278,15 @@ attn_prefill_tc2_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap kv
         for (int j = 0; ok && j < n_kt; ++j) {
           const bool more = j + 1 < n_kt;
           const Cur cv = ck.next(), cn = cv.next();
-          ok = wait_full(cv);
+          // V_j and K_(j+1) landed long ago as a rule: both tests go first, where the tensor pipe still works on S_B or waits
+          // for tile A's softmax anyway, and not between tile A's two MMA groups
+          ok = wait_full(cv) && (!more || wait_full(cn));
           if (ok && j < nA) {
             ok = wait_all(bar(C_PFULL + 0), ph_p[0]);
             ph_p[0] ^= 1u;
             if (ok) { tc_fence_after(); issue_pv(0, cv, j == 0, j == nA - 1); }
           }
-          if (ok && more) ok = wait_full(cn);
           if (!ok) break;
-          tc_fence_after();
           if (j + 1 < nA) issue_s(0, cn);
           if (j < nB) {
             ok = wait_all(bar(C_PFULL + 1), ph_p[1]);
